@@ -1,0 +1,149 @@
+"""Seeded synthetic attention workloads and their bookkeeping.
+
+This module only draws random tensors and counts work; it contains none of the
+attention arithmetic.  It is the one module that both the CUDA path's tests and
+the CPU oracle's tests may import.
+
+Generation rule (every workload): one CPU ``torch.Generator`` seeded with the
+workload's seed draws fp32 Q, then K, then V, in that order; the stated
+transform is applied in fp32; the result is rounded to bf16 (round to nearest
+even).  The shapes mirror the paper's evaluation of attention (Section 9:
+causal bf16 grouped-query prefill, head dimension 128, sequence lengths from
+1024 to 16384) plus a tiny case and a wide non-causal case.
+"""
+from __future__ import annotations
+
+import hashlib
+import math
+from dataclasses import dataclass, replace
+
+import torch
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    B: int
+    H: int
+    Hkv: int
+    Sq: int
+    Sk: int
+    D: int
+    causal: bool
+    seed: int
+    dist: str = "normal"          # "normal": N(0,1); "uniform": U[-2, 2]
+    peaked_every: int = 0          # >0: key rows j % peaked_every == 0 are multiplied by 4
+    note: str = ""
+
+    @property
+    def scale(self) -> float:
+        """1/sqrt(D), rounded to fp32 (the value handed to the library)."""
+        return float(torch.tensor(1.0 / math.sqrt(self.D), dtype=torch.float32).item())
+
+    @property
+    def G(self) -> int:
+        return self.H // self.Hkv
+
+
+WORKLOADS = {
+    "c1_tiny": Workload("c1_tiny", 1, 2, 2, 128, 128, 64, False, 0,
+                        note="tiny non-causal case the oracle finishes instantly"),
+    "c2_mha_prefill": Workload("c2_mha_prefill", 4, 32, 32, 2048, 2048, 128, True, 1,
+                               note="causal multi-head prefill"),
+    "c3_gqa_prefill": Workload("c3_gqa_prefill", 2, 64, 8, 4096, 4096, 128, True, 2,
+                               note="causal grouped-query prefill, 8 query heads per KV head"),
+    "c4_long_context": Workload("c4_long_context", 1, 32, 8, 16384, 16384, 128, True, 3,
+                                peaked_every=64,
+                                note="long causal prefill, every 64th key row x4 (peaked softmax rows)"),
+    "c5_wide_noncausal": Workload("c5_wide_noncausal", 8, 16, 16, 8192, 8192, 64, False, 4,
+                                  dist="uniform", note="encoder-style, head dim 64, U[-2,2]"),
+}
+
+# The paper's own attention workload (Section 9): causal bf16 GQA, batch 16,
+# 8 query heads, 1 KV head, head dimension 128, N in {1024..16384}.
+for _n in (1024, 2048, 4096, 8192, 16384):
+    WORKLOADS["paper_gqa_n%d" % _n] = Workload(
+        "paper_gqa_n%d" % _n, 16, 8, 1, _n, _n, 128, True, 100 + _n // 1024,
+        note="the paper's evaluation shape (LLaMA-3 70B prefill under 8-way TP)")
+
+
+def get(name: str) -> Workload:
+    return WORKLOADS[name]
+
+
+def small_variant(w: Workload, **kw) -> Workload:
+    """A same-recipe workload with some fields overridden (tests use this)."""
+    return replace(w, **kw)
+
+
+def make_inputs(w: Workload):
+    """(q, k, v) as CPU bf16 tensors [B,H,Sq,D], [B,Hkv,Sk,D], [B,Hkv,Sk,D]."""
+    g = torch.Generator(device="cpu")
+    g.manual_seed(w.seed)
+    shapes = [(w.B, w.H, w.Sq, w.D), (w.B, w.Hkv, w.Sk, w.D), (w.B, w.Hkv, w.Sk, w.D)]
+    out = []
+    for idx, shp in enumerate(shapes):
+        if w.dist == "normal":
+            x = torch.randn(shp, generator=g, dtype=torch.float32)
+        elif w.dist == "uniform":
+            x = torch.rand(shp, generator=g, dtype=torch.float32) * 4.0 - 2.0
+        else:
+            raise ValueError("unknown dist %r" % w.dist)
+        if idx == 1 and w.peaked_every > 0:
+            x[:, :, :: w.peaked_every, :] *= 4.0
+        out.append(x.to(torch.bfloat16))
+    return tuple(out)
+
+
+def tensor_sha256(t: torch.Tensor) -> str:
+    return hashlib.sha256(t.contiguous().view(torch.uint8).numpy().tobytes()).hexdigest()
+
+
+def visible_pairs(w: Workload) -> int:
+    """Number of (query, key) pairs the mask leaves visible, over all b, h."""
+    if not w.causal:
+        per_head = w.Sq * w.Sk
+    else:
+        off = w.Sk - w.Sq
+        per_head = sum(min(w.Sk, max(0, i + 1 + off)) for i in range(w.Sq))
+    return w.B * w.H * per_head
+
+
+def attn_flops(w: Workload) -> float:
+    """Counted FLOPs: 4*B*H*Sq*Sk*D, halved when causal."""
+    f = 4.0 * w.B * w.H * w.Sq * w.Sk * w.D
+    return f * 0.5 if w.causal else f
+
+
+def min_hbm_bytes(w: Workload) -> int:
+    """|Q| + |K| + |V| + |O| + |LSE| in bytes: every tensor touched once."""
+    q = w.B * w.H * w.Sq * w.D * 2
+    kv = 2 * w.B * w.Hkv * w.Sk * w.D * 2
+    o = q
+    lse = w.B * w.H * w.Sq * 4
+    return q + kv + o + lse
+
+
+def sample_rows(w: Workload, n_random: int, seed: int = 12345, tile: int = 128):
+    """Rows (b, h, i) for sampled parity on large workloads.
+
+    Every (b, h) contributes the rows next to each multiple of ``tile`` near
+    the start, middle and end; ``n_random`` further rows are uniform over
+    (b, h, i).
+    """
+    edge = set()
+    for base in (0, tile, 2 * tile, (w.Sq // 2 // tile) * tile, ((w.Sq - 1) // tile) * tile):
+        for d in (-1, 0, 1):
+            i = base + d
+            if 0 <= i < w.Sq:
+                edge.add(i)
+    edge.add(w.Sq - 1)
+    rows = [(b, h, i) for b in range(w.B) for h in range(w.H) for i in sorted(edge)]
+    g = torch.Generator(device="cpu")
+    g.manual_seed(seed)
+    if n_random > 0:
+        rb = torch.randint(0, w.B, (n_random,), generator=g)
+        rh = torch.randint(0, w.H, (n_random,), generator=g)
+        ri = torch.randint(0, w.Sq, (n_random,), generator=g)
+        rows += list(zip(rb.tolist(), rh.tolist(), ri.tolist()))
+    return rows
