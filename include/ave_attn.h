@@ -1,0 +1,110 @@
+/*
+ * ave_attn -- flash-attention forward for NVIDIA B200 (sm_100a), C ABI.
+ *
+ * Operation (paper Section 2: S = Q K^T, P = softmax_row(S), O = P V, tiled
+ * with an online softmax so S is never materialised; Fig. 1 for the
+ * grouped-query head mapping idx_h / gqa; Section 9 for the causal workload):
+ *
+ *   for every batch b, query head h, query row i, with g = h / (H / Hkv):
+ *     t_j  = scale * sum_d Q[b,h,i,d] * K[b,g,j,d]          j in [0, Sk)
+ *     key j is visible iff !causal or j <= i + (Sk - Sq)
+ *     LSE[b,h,i] = ln sum_{visible j} exp(t_j)               (natural log)
+ *     O[b,h,i,:] = sum_{visible j} exp(t_j - LSE) * V[b,g,j,:]
+ *   A row with no visible key gets O = 0 and LSE = -inf.
+ *
+ * Arithmetic: bf16 operands, fp32 accumulation on the tensor cores, fp32
+ * softmax statistics, probabilities rounded to bf16 for the second product,
+ * O rounded to bf16 (round to nearest even) once at the end.
+ *
+ * Every pointer named "device" must be dereferenceable by the current CUDA
+ * device; the caller owns all buffers and the stream.  Calls enqueue work on
+ * `stream` and return without synchronising; outputs are valid once the stream
+ * reaches that point.  Inputs are never written; outputs must not alias inputs.
+ * No call falls back to the CPU: without a compute-capability-10.0 device the
+ * launch entry points return AVE_ERR_UNSUPPORTED_DEVICE or AVE_ERR_CUDA.
+ */
+#ifndef AVE_ATTN_H
+#define AVE_ATTN_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    AVE_OK = 0,
+    AVE_ERR_NULL_POINTER = 1,       /* q, k, v, o or lse is NULL */
+    AVE_ERR_BAD_SHAPE = 2,          /* a size <= 0, H % Hkv != 0, or a size beyond the limits below */
+    AVE_ERR_UNSUPPORTED_D = 3,      /* D not in {64, 128} */
+    AVE_ERR_MISALIGNED = 4,         /* q, k, v, o not 16-byte aligned, or lse not 4-byte aligned */
+    AVE_ERR_BAD_SCALE = 5,          /* scale is NaN or infinite (zero and negative values are allowed) */
+    AVE_ERR_UNSUPPORTED_DEVICE = 6, /* the current device is not compute capability 10.x */
+    AVE_ERR_CUDA = 7,               /* a CUDA call failed; see ave_attn_last_cuda_error() */
+    AVE_ERR_DEVICE_TIMEOUT = 8,     /* a bounded wait inside a kernel gave up (ave_attn_device_status) */
+    AVE_ERR_WORKSPACE = 9           /* workspace NULL, misaligned or too small */
+} ave_status_t;
+
+/*
+ * Attention forward, definition at the top of this file (paper Section 2 and
+ * Fig. 1).  All pointers are DEVICE pointers to contiguous row-major tensors:
+ *   q   bf16 [B, H,   Sq, D]   read
+ *   k   bf16 [B, Hkv, Sk, D]   read
+ *   v   bf16 [B, Hkv, Sk, D]   read
+ *   o   bf16 [B, H,   Sq, D]   written
+ *   lse fp32 [B, H,   Sq]      written
+ * Limits: D in {64, 128}; H % Hkv == 0; Sq, Sk < 2^31 / 2; B * H < 2^31.
+ * causal: 0 = every key visible, nonzero = bottom-right aligned causal mask.
+ * scale: multiplies Q K^T before the softmax (callers normally pass 1/sqrt(D)).
+ * stream: a cudaStream_t; NULL is the legacy default stream.
+ * Arguments are validated in the order of ave_status_t before any CUDA call;
+ * on any error nothing is launched and the outputs are untouched.
+ * Returns an ave_status_t.
+ */
+int ave_attn_fwd(const void *q, const void *k, const void *v, void *o, float *lse,
+                 int B, int H, int Hkv, int Sq, int Sk, int D,
+                 int causal, float scale, void *stream);
+
+/*
+ * The same operation for tensors that live in HOST memory (same layouts and
+ * limits).  The call enqueues, on `stream`: host-to-device copies of q, k, v
+ * into `workspace`, the attention kernel, and device-to-host copies of o and
+ * lse.  `workspace` is a DEVICE buffer of at least
+ * ave_attn_host_workspace_bytes(...) bytes, 256-byte aligned, owned by the
+ * caller and reusable across calls on the same stream.  Copies are
+ * asynchronous only when the host buffers are page-locked; either way the
+ * results are valid after the stream has been synchronised.
+ */
+int ave_attn_fwd_host(const void *q_host, const void *k_host, const void *v_host,
+                      void *o_host, float *lse_host,
+                      int B, int H, int Hkv, int Sq, int Sk, int D,
+                      int causal, float scale,
+                      void *workspace, size_t workspace_bytes, void *stream);
+
+/* Bytes of device workspace ave_attn_fwd_host needs; 0 if the shape is invalid. */
+size_t ave_attn_host_workspace_bytes(int B, int H, int Hkv, int Sq, int Sk, int D);
+
+/*
+ * Synchronises the current device, then reads and clears the device-side
+ * status word that kernels set when one of their bounded waits (on an
+ * mbarrier) runs out.  Returns AVE_OK, AVE_ERR_DEVICE_TIMEOUT (with the raw
+ * word in *raw_word if it is not NULL), or AVE_ERR_CUDA.
+ */
+int ave_attn_device_status(unsigned int *raw_word);
+
+/* Number of kernels this library has launched in this process so far. */
+unsigned long long ave_attn_launch_count(void);
+
+/* Static, human-readable text for a status code. */
+const char *ave_attn_strerror(int status);
+
+/* Library version, major * 10000 + minor * 100 + patch. */
+int ave_attn_version(void);
+
+/* cudaError_t / CUresult of the last failing CUDA call on this thread. */
+int ave_attn_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

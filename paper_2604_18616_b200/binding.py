@@ -1,0 +1,157 @@
+"""ctypes binding of ``libave_attn.so``: argument marshalling only.
+
+Every function has the name and argument order of its C counterpart in
+``include/ave_attn.h``; tensors are passed as their ``data_ptr()``.  Nothing
+here computes: if the library has not been built the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libave_attn.so")
+
+AVE_OK = 0
+AVE_ERR_NULL_POINTER = 1
+AVE_ERR_BAD_SHAPE = 2
+AVE_ERR_UNSUPPORTED_D = 3
+AVE_ERR_MISALIGNED = 4
+AVE_ERR_BAD_SCALE = 5
+AVE_ERR_UNSUPPORTED_DEVICE = 6
+AVE_ERR_CUDA = 7
+AVE_ERR_DEVICE_TIMEOUT = 8
+AVE_ERR_WORKSPACE = 9
+
+_lib = None
+
+
+class AveAttnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: status %d (%s), cuda error %d" % (
+            where, status, strerror(status), last_cuda_error()))
+
+
+def lib() -> ctypes.CDLL:
+    """Load the CUDA library (built by ``paper_2604_18616_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                "%s is missing: build it with `python -m paper_2604_18616_b200.build` "
+                "(there is no CPU fallback)" % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        vp, ci, cf = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
+        L.ave_attn_fwd.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, cf, vp]
+        L.ave_attn_fwd.restype = ci
+        L.ave_attn_fwd_host.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, cf, vp, ctypes.c_size_t, vp]
+        L.ave_attn_fwd_host.restype = ci
+        L.ave_attn_host_workspace_bytes.argtypes = [ci] * 6
+        L.ave_attn_host_workspace_bytes.restype = ctypes.c_size_t
+        L.ave_attn_device_status.argtypes = [ctypes.POINTER(ctypes.c_uint)]
+        L.ave_attn_device_status.restype = ci
+        L.ave_attn_launch_count.argtypes = []
+        L.ave_attn_launch_count.restype = ctypes.c_ulonglong
+        L.ave_attn_strerror.argtypes = [ci]
+        L.ave_attn_strerror.restype = ctypes.c_char_p
+        L.ave_attn_version.argtypes = []
+        L.ave_attn_version.restype = ci
+        L.ave_attn_last_cuda_error.argtypes = []
+        L.ave_attn_last_cuda_error.restype = ci
+        _lib = L
+    return _lib
+
+
+def strerror(status: int) -> str:
+    return lib().ave_attn_strerror(int(status)).decode()
+
+
+def version() -> int:
+    return int(lib().ave_attn_version())
+
+
+def last_cuda_error() -> int:
+    return int(lib().ave_attn_last_cuda_error())
+
+
+def launch_count() -> int:
+    return int(lib().ave_attn_launch_count())
+
+
+def device_status():
+    """(status, raw word) after synchronising the device."""
+    raw = ctypes.c_uint(0)
+    st = lib().ave_attn_device_status(ctypes.byref(raw))
+    return int(st), int(raw.value)
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def ave_attn_fwd_raw(q_ptr, k_ptr, v_ptr, o_ptr, lse_ptr, B, H, Hkv, Sq, Sk, D, causal, scale, stream_ptr=None) -> int:
+    """The C call with plain integers for pointers; returns the status code."""
+    return int(lib().ave_attn_fwd(
+        ctypes.c_void_p(q_ptr), ctypes.c_void_p(k_ptr), ctypes.c_void_p(v_ptr),
+        ctypes.c_void_p(o_ptr), ctypes.c_void_p(lse_ptr),
+        B, H, Hkv, Sq, Sk, D, int(bool(causal)), float(scale), ctypes.c_void_p(stream_ptr)))
+
+
+def ave_attn_fwd(q, k, v, o=None, lse=None, causal=False, scale=None, stream=None):
+    """O, LSE = attention(q, k, v) on the tensors' CUDA device.
+
+    q [B,H,Sq,D], k/v [B,Hkv,Sk,D]: contiguous CUDA bf16.  ``o`` (bf16) and
+    ``lse`` (fp32) are allocated when not given.  Raises ``AveAttnError`` on a
+    non-zero status.
+    """
+    for t in (q, k, v):
+        if not (t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous() and t.dim() == 4):
+            raise ValueError("q, k, v must be contiguous 4-D CUDA bfloat16 tensors")
+    B, H, Sq, D = q.shape
+    Bk, Hkv, Sk, Dk = k.shape
+    if tuple(v.shape) != tuple(k.shape) or Bk != B or Dk != D:
+        raise ValueError("inconsistent q/k/v shapes")
+    if o is None:
+        o = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((B, H, Sq), dtype=torch.float32, device=q.device)
+    if scale is None:
+        scale = D ** -0.5
+    with torch.cuda.device(q.device):
+        st = lib().ave_attn_fwd(
+            ctypes.c_void_p(q.data_ptr()), ctypes.c_void_p(k.data_ptr()), ctypes.c_void_p(v.data_ptr()),
+            ctypes.c_void_p(o.data_ptr()), ctypes.c_void_p(lse.data_ptr()),
+            B, H, Hkv, Sq, Sk, D, int(bool(causal)), float(scale), _stream_ptr(stream))
+    if st != AVE_OK:
+        raise AveAttnError(st, "ave_attn_fwd")
+    return o, lse
+
+
+def host_workspace_bytes(B, H, Hkv, Sq, Sk, D) -> int:
+    return int(lib().ave_attn_host_workspace_bytes(B, H, Hkv, Sq, Sk, D))
+
+
+def ave_attn_fwd_host(q, k, v, o, lse, workspace, causal=False, scale=None, stream=None):
+    """Host-buffer variant: q, k, v, o, lse are CPU tensors (pinned for
+    asynchronous copies), ``workspace`` a CUDA uint8 tensor of at least
+    ``host_workspace_bytes`` bytes.  Results are valid after the stream has
+    been synchronised."""
+    B, H, Sq, D = q.shape
+    _, Hkv, Sk, _ = k.shape
+    if scale is None:
+        scale = D ** -0.5
+    with torch.cuda.device(workspace.device):
+        st = lib().ave_attn_fwd_host(
+            ctypes.c_void_p(q.data_ptr()), ctypes.c_void_p(k.data_ptr()), ctypes.c_void_p(v.data_ptr()),
+            ctypes.c_void_p(o.data_ptr()), ctypes.c_void_p(lse.data_ptr()),
+            B, H, Hkv, Sq, Sk, D, int(bool(causal)), float(scale),
+            ctypes.c_void_p(workspace.data_ptr()), ctypes.c_size_t(workspace.numel() * workspace.element_size()),
+            _stream_ptr(stream))
+    if st != AVE_OK:
+        raise AveAttnError(st, "ave_attn_fwd_host")
+    return o, lse

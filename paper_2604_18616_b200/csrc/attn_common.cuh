@@ -1,0 +1,79 @@
+// Shared definitions of the attention-forward kernels: tile sizes, kernel
+// parameters, tcgen05 descriptor encodings, bounded mbarrier waits.
+#pragma once
+
+#include <cstdint>
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "ptx_sm100.cuh"
+
+namespace ave {
+
+constexpr int BM = 128;  // query rows per MMA tile (= TMEM lanes)
+constexpr int BN = 128;  // keys per step
+
+// Device-side status word; a kernel ORs a code in when a bounded wait gives up.
+// (This header is included by exactly one translation unit.)
+__device__ unsigned int g_device_status = 0;
+
+constexpr unsigned int STATUS_TIMEOUT_LOAD = 1u;     // waiting for a TMA load
+constexpr unsigned int STATUS_TIMEOUT_MMA = 2u;      // waiting for a tcgen05.commit
+constexpr unsigned int STATUS_TIMEOUT_SOFTMAX = 4u;  // MMA warp waiting for P
+constexpr unsigned int STATUS_TIMEOUT_SLOT = 8u;     // producer waiting for a free stage
+
+// Upper bound on mbarrier polls before a wait is abandoned (a fraction of a
+// second; legitimate waits last microseconds).
+constexpr uint32_t WAIT_LIMIT = 1u << 23;
+
+struct FwdParams {
+    void *o;          // bf16 [B, H, Sq, D]
+    float *lse;       // fp32 [B, H, Sq]
+    int H, Hkv;       // query heads, key/value heads
+    int Sq, Sk;       // sequence lengths
+    int n_qblk;       // query blocks per (b, h)
+    int total_blocks; // n_qblk * B * H
+    float scale_log2; // scale * log2(e)
+};
+
+// tcgen05 instruction descriptor, kind::f16: fp32 accumulator, bf16 A and B,
+// A K-major (or in TMEM), B K-major (b_mn_major = 0) or MN-major (= 1).
+__host__ __device__ constexpr uint32_t make_idesc_bf16(int m, int n, int b_mn_major) {
+    return (1u << 4)                         // D format: f32
+           | (1u << 7)                       // A format: bf16
+           | (1u << 10)                      // B format: bf16
+           | (0u << 15)                      // A major: K
+           | (uint32_t(b_mn_major) << 16)    // B major
+           | (uint32_t(n >> 3) << 17)        // N / 8
+           | (uint32_t(m >> 4) << 24);       // M / 16
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, without the address.
+//   K-major operand  (rows of 64 bf16 = 128 B, 8-row atoms of 1024 B):
+//       lbo unused (16), sbo = 1024 (next 8 rows)
+//   MN-major operand (64 contiguous bf16 along MN per K row of 128 B):
+//       lbo = bytes between 64-wide MN groups, sbo = 1024 (next 8 K rows)
+__host__ __device__ constexpr uint64_t make_sdesc_sw128(uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return (uint64_t((lbo_bytes >> 4) & 0x3FFFu) << 16) | (uint64_t((sbo_bytes >> 4) & 0x3FFFu) << 32) |
+           (1ull << 46)    // descriptor version for sm_100
+           | (2ull << 61); // swizzle mode: 128 B
+}
+__device__ __forceinline__ uint64_t sdesc_at(uint64_t desc_no_addr, uint32_t smem_addr) {
+    return desc_no_addr | uint64_t((smem_addr >> 4) & 0x3FFFu);
+}
+
+// Poll an mbarrier phase with an iteration limit.  Returns false when the
+// limit was reached or another thread of the CTA has already given up;
+// `abort_flag` is a shared-memory word all roles watch.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                                  unsigned int code) {
+    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 0x3FFu) == 0x3FFu && *abort_flag != 0) return false;
+    }
+    *abort_flag = 1;
+    atomicOr(&g_device_status, code);
+    return false;
+}
+
+}  // namespace ave
