@@ -1,0 +1,98 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports
+every function the header declares, and validates arguments before touching
+CUDA."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2604_18616_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build_cuda()
+    return binding.lib()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "ave_attn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ave_attn_\w+)\s*\(", text)))
+
+
+def test_header_declares_the_expected_entry_points():
+    names = declared_functions()
+    for n in ("ave_attn_fwd", "ave_attn_fwd_host", "ave_attn_host_workspace_bytes", "ave_attn_device_status",
+              "ave_attn_launch_count", "ave_attn_strerror", "ave_attn_version", "ave_attn_last_cuda_error"):
+        assert n in names
+
+
+def test_library_exports_every_declared_symbol(lib):
+    raw = ctypes.CDLL(binding.LIB_PATH)
+    for n in declared_functions():
+        assert hasattr(raw, n), "libave_attn.so does not export %s" % n
+
+
+def test_version_and_strerror(lib):
+    assert binding.version() >= 100
+    seen = set()
+    for code in range(0, 10):
+        msg = binding.strerror(code)
+        assert msg and msg != "unknown status"
+        seen.add(msg)
+    assert len(seen) == 10
+    assert binding.strerror(12345) == "unknown status"
+
+
+def test_validation_order_before_any_cuda_call(lib):
+    A = 4096  # aligned fake address: validation must reject before dereferencing anything
+    f = binding.ave_attn_fwd_raw
+    assert f(0, A, A, A, A, 1, 2, 2, 128, 128, 64, 0, 1.0) == binding.AVE_ERR_NULL_POINTER
+    assert f(A, A, A, A, 0, 1, 2, 2, 128, 128, 64, 0, 1.0) == binding.AVE_ERR_NULL_POINTER
+    assert f(A, A, A, A, A, 0, 2, 2, 128, 128, 64, 0, 1.0) == binding.AVE_ERR_BAD_SHAPE
+    assert f(A, A, A, A, A, 1, 2, 2, -5, 128, 64, 0, 1.0) == binding.AVE_ERR_BAD_SHAPE
+    assert f(A, A, A, A, A, 1, 6, 4, 128, 128, 64, 0, 1.0) == binding.AVE_ERR_BAD_SHAPE      # H % Hkv
+    assert f(A, A, A, A, A, 1, 2, 2, 1 << 30, 128, 64, 0, 1.0) == binding.AVE_ERR_BAD_SHAPE
+    assert f(A, A, A, A, A, 1, 2, 2, 128, 128, 96, 0, 1.0) == binding.AVE_ERR_UNSUPPORTED_D
+    assert f(A, A, A, A, A, 1, 2, 2, 128, 128, 256, 0, 1.0) == binding.AVE_ERR_UNSUPPORTED_D
+    assert f(A + 8, A, A, A, A, 1, 2, 2, 128, 128, 64, 0, 1.0) == binding.AVE_ERR_MISALIGNED
+    assert f(A, A, A, A + 2, A, 1, 2, 2, 128, 128, 64, 0, 1.0) == binding.AVE_ERR_MISALIGNED
+    assert f(A, A, A, A, A + 2, 1, 2, 2, 128, 128, 64, 0, 1.0) == binding.AVE_ERR_MISALIGNED
+    assert f(A, A, A, A, A, 1, 2, 2, 128, 128, 64, 0, float("inf")) == binding.AVE_ERR_BAD_SCALE
+    assert f(A, A, A, A, A, 1, 2, 2, 128, 128, 64, 0, float("nan")) == binding.AVE_ERR_BAD_SCALE
+    # bad D outranks misalignment, bad shape outranks bad D (order of the status codes)
+    assert f(A + 8, A, A, A, A, 1, 2, 2, 128, 128, 96, 0, 1.0) == binding.AVE_ERR_UNSUPPORTED_D
+    assert f(A, A, A, A, A, 1, 3, 2, 128, 128, 96, 0, 1.0) == binding.AVE_ERR_BAD_SHAPE
+
+
+def test_no_silent_cpu_fallback_without_a_device(lib):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a CUDA device is present")
+    A = 4096
+    st = binding.ave_attn_fwd_raw(A, A, A, A, A, 1, 2, 2, 128, 128, 64, 0, 1.0)
+    assert st in (binding.AVE_ERR_CUDA, binding.AVE_ERR_UNSUPPORTED_DEVICE)
+    assert binding.launch_count() == 0
+
+
+def test_host_workspace_bytes(lib):
+    n = binding.host_workspace_bytes(4, 32, 32, 2048, 2048, 128)
+    q = 4 * 32 * 2048 * 128 * 2
+    assert n == 4 * q + 4 * 32 * 2048 * 4
+    assert binding.host_workspace_bytes(1, 3, 2, 8, 8, 64) == 0      # invalid shape
+    assert binding.host_workspace_bytes(1, 2, 2, 8, 8, 32) == 0      # unsupported D
+    assert binding.host_workspace_bytes(1, 1, 1, 1, 1, 64) == 256 * 5  # each buffer rounded up to 256 B
+
+
+def test_host_entry_point_validates_workspace(lib):
+    A = 4096
+    L = binding.lib()
+    vp = ctypes.c_void_p
+    st = L.ave_attn_fwd_host(vp(A), vp(A), vp(A), vp(A), vp(A), 1, 2, 2, 128, 128, 64, 0, 1.0, vp(0), 0, vp(0))
+    assert st == binding.AVE_ERR_WORKSPACE
+    st = L.ave_attn_fwd_host(vp(A), vp(A), vp(A), vp(A), vp(A), 1, 2, 2, 128, 128, 64, 0, 1.0, vp(A), 16, vp(0))
+    assert st == binding.AVE_ERR_WORKSPACE
