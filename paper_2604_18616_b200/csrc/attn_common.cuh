@@ -24,7 +24,7 @@ constexpr unsigned int STATUS_TIMEOUT_SLOT = 8u;     // producer waiting for a f
 
 // Upper bound on mbarrier polls before a wait is abandoned (a fraction of a
 // second; legitimate waits last microseconds).
-constexpr uint32_t WAIT_LIMIT = 1u << 23;
+constexpr uint32_t WAIT_LIMIT = 1u << 21;
 
 struct FwdParams {
     void *o;          // bf16 [B, H, Sq, D]

@@ -12,7 +12,7 @@
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 
-#include "attn_fwd_simple.cuh"
+#include "attn_fwd_ws.cuh"
 
 namespace {
 
@@ -106,10 +106,10 @@ int check_device() {
 }
 
 template <int D, bool CAUSAL>
-int launch_simple(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const ave::FwdParams &p,
-                  cudaStream_t stream) {
-    using Cfg = ave::SimpleCfg<D>;
-    auto kern = ave::attn_fwd_simple_kernel<D, CAUSAL>;
+int launch_ws(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const CUtensorMap &to,
+              const ave::FwdParams &p, cudaStream_t stream) {
+    using Cfg = ave::WsCfg<D>;
+    auto kern = ave::attn_fwd_ws_kernel<D, CAUSAL>;
     static std::atomic<bool> configured{false};  // per instantiation
     if (!configured.load(std::memory_order_acquire)) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
@@ -119,7 +119,7 @@ int launch_simple(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMa
         }
         configured.store(true, std::memory_order_release);
     }
-    kern<<<dim3(p.total_blocks), dim3(Cfg::kThreads), Cfg::kSmemBytes, stream>>>(tq, tk, tv, p);
+    kern<<<dim3(p.total_blocks), dim3(Cfg::kThreads), Cfg::kSmemBytes, stream>>>(tq, tk, tv, to, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
         t_last_cuda_error = int(e);
@@ -142,8 +142,9 @@ int ave_attn_fwd(const void *q, const void *k, const void *v, void *o, float *ls
     st = check_device();
     if (st != AVE_OK) return st;
 
-    CUtensorMap tq, tk, tv;
+    CUtensorMap tq, tk, tv, to;
     if (!encode_map(&tq, q, D, Sq, (long long)B * H, ave::BM)) return AVE_ERR_CUDA;
+    if (!encode_map(&to, o, D, Sq, (long long)B * H, ave::BM)) return AVE_ERR_CUDA;
     if (!encode_map(&tk, k, D, Sk, (long long)B * Hkv, ave::BN)) return AVE_ERR_CUDA;
     if (!encode_map(&tv, v, D, Sk, (long long)B * Hkv, ave::BN)) return AVE_ERR_CUDA;
 
@@ -154,13 +155,14 @@ int ave_attn_fwd(const void *q, const void *k, const void *v, void *o, float *ls
     p.Hkv = Hkv;
     p.Sq = Sq;
     p.Sk = Sk;
-    p.n_qblk = (Sq + ave::BM - 1) / ave::BM;
+    p.n_qblk = (Sq + 2 * ave::BM - 1) / (2 * ave::BM);
     p.total_blocks = p.n_qblk * B * H;
     p.scale_log2 = scale * 1.4426950408889634f;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (D == 128) return causal ? launch_simple<128, true>(tq, tk, tv, p, s) : launch_simple<128, false>(tq, tk, tv, p, s);
-    return causal ? launch_simple<64, true>(tq, tk, tv, p, s) : launch_simple<64, false>(tq, tk, tv, p, s);
+    if (D == 128)
+        return causal ? launch_ws<128, true>(tq, tk, tv, to, p, s) : launch_ws<128, false>(tq, tk, tv, to, p, s);
+    return causal ? launch_ws<64, true>(tq, tk, tv, to, p, s) : launch_ws<64, false>(tq, tk, tv, to, p, s);
 }
 
 size_t ave_attn_host_workspace_bytes(int B, int H, int Hkv, int Sq, int Sk, int D) {
