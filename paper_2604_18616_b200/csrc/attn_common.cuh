@@ -31,8 +31,10 @@ struct FwdParams {
     float *lse;       // fp32 [B, H, Sq]
     int H, Hkv;       // query heads, key/value heads
     int Sq, Sk;       // sequence lengths
-    int n_qblk;       // query blocks per (b, h)
-    int total_blocks; // n_qblk * B * H
+    int BH;           // B * H
+    int n_qblk;       // work tiles (blocks of 256 query rows) per (b, h)
+    int total_blocks; // n_qblk * BH = grid size
+    int heads_per_group;  // (b, h) pairs whose work tiles are launched together (their K/V share L2)
     float scale_log2; // scale * log2(e)
 };
 
@@ -62,6 +64,18 @@ __device__ __forceinline__ uint64_t sdesc_at(uint64_t desc_no_addr, uint32_t sme
     return desc_no_addr | uint64_t((smem_addr >> 4) & 0x3FFFu);
 }
 
+// Optional role timeline (builds with -DAVE_TRACE=<cta index> only): SM clock
+// stamps of one CTA, [role][iteration][slot], read back by a debug entry point.
+#ifdef AVE_TRACE
+constexpr int TRACE_ROLES = 4, TRACE_ITERS = 64, TRACE_SLOTS = 8;
+__device__ long long g_trace[TRACE_ROLES][TRACE_ITERS][TRACE_SLOTS];
+__device__ __forceinline__ void trace_stamp(int role, int iter, int slot) {
+    if (blockIdx.x == AVE_TRACE && iter < TRACE_ITERS) g_trace[role][iter][slot] = clock64();
+}
+#else
+__device__ __forceinline__ void trace_stamp(int, int, int) {}
+#endif
+
 // Poll an mbarrier phase with an iteration limit.  Returns false when the
 // limit was reached or another thread of the CTA has already given up;
 // `abort_flag` is a shared-memory word all roles watch.
@@ -70,6 +84,21 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
     for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 0x3FFu) == 0x3FFu && *abort_flag != 0) return false;
+    }
+    *abort_flag = 1;
+    atomicOr(&g_device_status, code);
+    return false;
+}
+
+// The same with a non-suspending poll: the waiter notices the completion within a
+// few tens of cycles instead of after a wake-up, at the price of issue slots.
+// For the one warp whose reaction time is on the critical path.
+constexpr uint32_t SPIN_LIMIT = 1u << 25;
+__device__ __forceinline__ bool mbar_spin_bounded(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                                  unsigned int code) {
+    for (uint32_t it = 0; it < SPIN_LIMIT; ++it) {
+        if (mbar_test_wait(bar, parity)) return true;
+        if ((it & 0xFFFFu) == 0xFFFFu && *abort_flag != 0) return false;
     }
     *abort_flag = 1;
     atomicOr(&g_device_status, code);

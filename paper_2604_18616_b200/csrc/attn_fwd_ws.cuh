@@ -1,15 +1,21 @@
-// Attention forward, warp-specialised kernel for sm_100a.
+// Attention forward, persistent warp-specialised kernel for sm_100a.
 //
-// One CTA owns a block of 256 query rows of one (batch, head): two 128-row
+// A work tile is a block of 256 query rows of one (batch, head): two 128-row
 // sub-tiles that ping-pong so the tensor pipe works on one while the softmax
 // of the other runs (the paper's "+Pipe": software pipelining across disjoint
 // groups of warps, Section 9; steps of the loop as in Section 2 / Fig. 1).
+// The grid has one CTA per work tile, ordered so that tiles sharing K/V run
+// together and long causal tiles come first; a CTA that finishes its tile
+// takes over a not-yet-started CTA's tile through cluster launch control, so
+// the resident CTAs persist and prefetch their next tile while finishing the
+// current one.
 //
-//   warp 0        producer: TMA loads of Q (once) and of the K/V ring
+//   warp 0        producer: TMA loads of Q and of the K/V ring
 //   warp 1        MMA issuer: S_t = Q_t K_j^T and O_t += P_t V_j on tcgen05
 //   warp 2        TMEM allocation / release
-//   warps 4..7    softmax of sub-tile 0 (one thread per query row)
-//   warps 8..11   softmax of sub-tile 1
+//   warp 3        tile scheduler (cluster launch control)
+//   warps 4..7    softmax + epilogue of sub-tile 0 (one thread per query row)
+//   warps 8..11   softmax + epilogue of sub-tile 1
 //
 // TMEM columns: S0 [0,128) S1 [128,256) O0 [256,256+D) O1 [384,384+D); P_t
 // (bf16 pairs) overwrites the first 64 columns of S_t once a thread holds its
@@ -17,28 +23,40 @@
 #pragma once
 
 #include "attn_common.cuh"
+#include "softmax_math.cuh"
 
 namespace ave {
 
 template <int D>
 struct WsCfg {
     static constexpr int kThreads = 384;
-    static constexpr int kQRows = 2 * BM;                    // query rows per CTA
+    static constexpr int kQRows = 2 * BM;                    // query rows per work tile
     static constexpr int kTileBytes = BM * D * 2;            // one Q sub-tile, K tile or V tile
-    static constexpr int kBoxBytes = BM * 64 * 2;            // one 64-column TMA box
+    static constexpr int kBoxBytes = BM * 64 * 2;            // one 64-column TMA box (128 rows x 128 B)
     static constexpr int kBoxes = D / 64;
-    static constexpr int kStages = (D == 128) ? 5 : 8;       // ring slots, K and V tiles alternate
-    static constexpr int kSmemBytes = kTileBytes * (2 + kStages) + 1024;
+    static constexpr int kStages = (D == 128) ? 4 : 8;       // ring slots, K and V tiles alternate
+    static constexpr int kStageOBytes = kBoxBytes;           // O staging per sub-tile: 64 columns at a time
+    static constexpr int kOutBoxRows = 32;                   // each softmax warp stores its own 32 rows
+    static constexpr int kSmemBytes = kTileBytes * (2 + kStages) + 2 * kStageOBytes + 1024;
     static constexpr uint32_t kTmemCols = 512;
     static constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO0 = 256, kColO1 = 384;
-    static constexpr int kRegsLight = 64;                    // producer / MMA warpgroup
+    static constexpr int kRegsLight = 64;                    // producer / MMA / scheduler warpgroup
     static constexpr int kRegsSoftmax = 216;                 // softmax warpgroups
+    static constexpr int kTileConsumers = 10;                // producer + MMA + 8 softmax warps read each tile id
 };
 
 // Rescale O only when the running maximum moved by more than this many
 // powers of two; until then probabilities are taken relative to a stale
 // maximum (at most 2^8 too large), which the final division by l undoes.
 constexpr float kRescaleThreshold = 8.0f;
+
+// Of every 8 consecutive pairs of probabilities, the pairs whose bit is set
+// here are exponentiated on the FMA pipe (exp2_fma_pipe) instead of the
+// exponential unit.
+#ifndef AVE_FMA_EXP_MASK
+#define AVE_FMA_EXP_MASK 0x00
+#endif
+constexpr unsigned kFmaPipeExpMask = AVE_FMA_EXP_MASK;
 
 template <int N>
 __device__ __forceinline__ void setmaxnreg_inc() {
@@ -48,9 +66,14 @@ template <int N>
 __device__ __forceinline__ void setmaxnreg_dec() {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
 }
-__device__ __forceinline__ void named_barrier_sync(int id, int nthreads) {
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
-}
+
+// One work tile, decoded from its position in the launch order.
+struct WorkTile {
+    int bh;      // b * H + h
+    int bg;      // b * Hkv + h / (H / Hkv): key/value head (Fig. 1: idx_h / gqa)
+    int q0;      // first query row
+    int n0, n1;  // key tiles the two sub-tiles visit (n1 >= n0)
+};
 
 // Number of key tiles a 128-row sub-tile starting at row i0 must visit.
 template <bool CAUSAL>
@@ -63,6 +86,53 @@ __device__ __forceinline__ int kv_tiles_for(int i0, int Sq, int Sk) {
     return n;
 }
 
+// Launch order: (batch, head) pairs in groups of p.heads_per_group (whose K/V
+// fit in L2 together); inside a group all heads' blocks of one query position,
+// longest (causal: last) position first.
+template <bool CAUSAL>
+__device__ __forceinline__ WorkTile decode_tile(int id, const FwdParams &p) {
+    const int per_group = p.heads_per_group * p.n_qblk;
+    const int grp = id / per_group;
+    const int rem = id - grp * per_group;
+    const int bh0 = grp * p.heads_per_group;
+    const int hg = min(p.heads_per_group, p.BH - bh0);
+    const int rank = rem / hg;
+    WorkTile w;
+    w.bh = bh0 + (rem - rank * hg);
+    const int qb = CAUSAL ? (p.n_qblk - 1 - rank) : rank;
+    const int b = w.bh / p.H;
+    const int h = w.bh - b * p.H;
+    w.bg = b * p.Hkv + h / (p.H / p.Hkv);
+    w.q0 = qb * 2 * BM;
+    w.n0 = kv_tiles_for<CAUSAL>(w.q0, p.Sq, p.Sk);
+    w.n1 = kv_tiles_for<CAUSAL>(w.q0 + BM, p.Sq, p.Sk);
+    return w;
+}
+
+// ---- cluster launch control: take over the tile of a CTA that has not started
+__device__ __forceinline__ void clc_try_cancel(uint32_t response_smem, uint32_t bar) {
+    asm volatile("clusterlaunchcontrol.try_cancel.async.shared::cta.mbarrier::complete_tx::bytes.b128 [%0], [%1];"
+                 ::"r"(response_smem), "r"(bar) : "memory");
+}
+// Decode a 16-byte response: the cancelled CTA's blockIdx.x, or -1 if nothing was cancelled.
+__device__ __forceinline__ int clc_decode(const volatile unsigned long long *response) {
+    const unsigned long long lo = response[0], hi = response[1];
+    uint32_t ok, x;
+    asm volatile(
+        "{\n"
+        ".reg .b128 resp;\n"
+        ".reg .pred p;\n"
+        "mov.b128 resp, {%2, %3};\n"
+        "clusterlaunchcontrol.query_cancel.is_canceled.pred.b128 p, resp;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "mov.u32 %1, 0;\n"
+        "@p clusterlaunchcontrol.query_cancel.get_first_ctaid::x.b32.b128 %1, resp;\n"
+        "}\n"
+        : "=r"(ok), "=r"(x)
+        : "l"(lo), "l"(hi));
+    return ok ? int(x) : -1;
+}
+
 template <int D, bool CAUSAL>
 __global__ void __launch_bounds__(384, 1)
 attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -71,8 +141,10 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     using Cfg = WsCfg<D>;
     constexpr int NS = Cfg::kStages;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bar_q[2], bar_s[2], bar_p[2], bar_o[2], bar_drain;
+    __shared__ __align__(16) unsigned long long clc_response[2][2];
+    __shared__ __align__(8) uint64_t bar_q_full[2], bar_q_empty[2], bar_s[2], bar_p[2], bar_o[2], bar_o_free[2];
     __shared__ __align__(8) uint64_t bar_full[NS], bar_empty[NS];
+    __shared__ __align__(8) uint64_t bar_tile_full[2], bar_tile_empty[2], bar_drain;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
@@ -80,19 +152,10 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     const int warp = tid >> 5;
     const int lane = tid & 31;
 
-    // ---- work decomposition (Fig. 1: grid = (q-block, head)); long causal blocks first
-    const int bh = blockIdx.x / p.n_qblk;
-    const int qb = p.n_qblk - 1 - (blockIdx.x % p.n_qblk);
-    const int b = bh / p.H;
-    const int h = bh - b * p.H;
-    const int bg = b * p.Hkv + h / (p.H / p.Hkv);  // key/value head: idx_h / gqa
-    const int q0 = qb * Cfg::kQRows;
-    const int n0 = kv_tiles_for<CAUSAL>(q0, p.Sq, p.Sk);
-    const int n1 = kv_tiles_for<CAUSAL>(q0 + BM, p.Sq, p.Sk);  // n1 >= n0
-
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t sQ = smem_base;                           // two sub-tiles
-    const uint32_t sRing = smem_base + 2 * Cfg::kTileBytes;  // NS slots
+    const uint32_t sQ = smem_base;                                   // two sub-tiles
+    const uint32_t sRing = sQ + 2 * Cfg::kTileBytes;                 // NS slots
+    const uint32_t sStage = sRing + NS * Cfg::kTileBytes;            // O staging, one box per sub-tile
 
     if (tid == 0) {
         // A wait that ran out earlier (in this launch or a previous one) leaves the
@@ -100,10 +163,14 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         // instead of each running into the same limit.
         abort_flag = (*reinterpret_cast<volatile unsigned int *>(&g_device_status) != 0) ? 1 : 0;
         for (int t = 0; t < 2; ++t) {
-            mbar_init(smem_u32(&bar_q[t]), 1);
+            mbar_init(smem_u32(&bar_q_full[t]), 1);
+            mbar_init(smem_u32(&bar_q_empty[t]), 1);
             mbar_init(smem_u32(&bar_s[t]), 1);
-            mbar_init(smem_u32(&bar_p[t]), 4);  // one arrival per softmax warp
+            mbar_init(smem_u32(&bar_p[t]), 4);       // one arrival per softmax warp
             mbar_init(smem_u32(&bar_o[t]), 1);
+            mbar_init(smem_u32(&bar_o_free[t]), 4);  // one arrival per softmax warp
+            mbar_init(smem_u32(&bar_tile_full[t]), 1);
+            mbar_init(smem_u32(&bar_tile_empty[t]), Cfg::kTileConsumers);
         }
         mbar_init(smem_u32(&bar_drain), 1);
         for (int s = 0; s < NS; ++s) {
@@ -122,42 +189,104 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     const uint32_t tmem = tmem_base_slot;
     const bool poisoned = abort_flag != 0;
 
+    // A full warp waits on an mbarrier phase; the verdict is made warp-uniform.
+    auto wait_bar = [&](uint64_t *bar, uint32_t parity, unsigned code) -> bool {
+        const bool r = mbar_wait_bounded(smem_u32(bar), parity, &abort_flag, code);
+        return __all_sync(0xffffffffu, r);
+    };
+    auto spin_bar = [&](uint64_t *bar, uint32_t parity, unsigned code) -> bool {
+        const bool r = mbar_spin_bounded(smem_u32(bar), parity, &abort_flag, code);
+        return __all_sync(0xffffffffu, r);
+    };
+    // Every consumer warp of the tile sequence calls this at the end of its n-th
+    // tile to learn the next one (-1: none left); one lane releases the slot.
+    auto next_tile = [&](int n, bool &ok) -> int {
+        const int slot = n & 1;
+        ok = wait_bar(&bar_tile_full[slot], (n >> 1) & 1, STATUS_TIMEOUT_SLOT);
+        if (!ok) return -1;
+        const int id = clc_decode(clc_response[slot]);
+        fence_proxy_async_smem();  // order the read before the slot's next asynchronous write
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bar_tile_empty[slot]));
+        return id;
+    };
+
     if (poisoned) {
         // nothing: fall through to the common exit
     } else if (warp < 4) {
         setmaxnreg_dec<Cfg::kRegsLight>();
-        if (warp == 0 && lane == 0 && n1 > 0) {
-            // =============================== producer ===============================
-            tma_prefetch_desc(&tm_q);
-            tma_prefetch_desc(&tm_k);
-            tma_prefetch_desc(&tm_v);
-            for (int t = 0; t < 2; ++t) {
-                const uint32_t bar = smem_u32(&bar_q[t]);
-                mbar_arrive_expect_tx(bar, Cfg::kTileBytes);
-                for (int x = 0; x < Cfg::kBoxes; ++x)
-                    tma_load_3d(sQ + t * Cfg::kTileBytes + x * Cfg::kBoxBytes, &tm_q, bar, x * 64, q0 + t * BM, bh);
-            }
-            int issued = 0;
+        if (warp == 3) {
+            // =============================== tile scheduler ===============================
+            const bool leader = elect_one();
             bool ok = true;
-            for (int it = 0; it < 2 * n1 && ok; ++it) {  // it even: K_{it/2}; odd: V_{it/2}
-                const int slot = it % NS, round = it / NS;
-                if (round > 0)
-                    ok = mbar_wait_bounded(smem_u32(&bar_empty[slot]), (round - 1) & 1, &abort_flag, STATUS_TIMEOUT_SLOT);
+            for (int k = 0; ok; ++k) {
+                const int slot = k & 1;
+                if (k >= 2) {  // every consumer has read the response this slot held two requests ago
+                    ok = wait_bar(&bar_tile_empty[slot], ((k >> 1) - 1) & 1, STATUS_TIMEOUT_SLOT);
+                    if (!ok) break;
+                }
+                if (leader) {
+                    mbar_arrive_expect_tx(smem_u32(&bar_tile_full[slot]), 16);
+                    clc_try_cancel(smem_u32(&clc_response[slot][0]), smem_u32(&bar_tile_full[slot]));
+                }
+                ok = wait_bar(&bar_tile_full[slot], (k >> 1) & 1, STATUS_TIMEOUT_SLOT);
                 if (!ok) break;
-                const uint32_t bar = smem_u32(&bar_full[slot]);
-                const CUtensorMap *tm = (it & 1) ? &tm_v : &tm_k;
-                mbar_arrive_expect_tx(bar, Cfg::kTileBytes);
-                for (int x = 0; x < Cfg::kBoxes; ++x)
-                    tma_load_3d(sRing + slot * Cfg::kTileBytes + x * Cfg::kBoxBytes, tm, bar, x * 64, (it >> 1) * BN, bg);
-                issued = it + 1;
+                if (clc_decode(clc_response[slot]) < 0) break;  // nothing left to take over: never ask again
+            }
+        } else if (warp == 0) {
+            // =============================== producer ===============================
+            const bool leader = elect_one();
+            if (leader) {
+                tma_prefetch_desc(&tm_q);
+                tma_prefetch_desc(&tm_k);
+                tma_prefetch_desc(&tm_v);
+            }
+            int ring = 0;  // K/V tiles loaded so far (ring position)
+            bool ok = true;
+            int id = blockIdx.x;
+            for (int n = 0; id >= 0 && ok; ++n) {
+                const WorkTile w = decode_tile<CAUSAL>(id, p);
+                for (int t = 0; t < 2 && ok; ++t) {
+                    if (n > 0) {  // the previous tile's last Q_t K^T has finished reading this buffer
+                        ok = wait_bar(&bar_q_empty[t], (n - 1) & 1, STATUS_TIMEOUT_SLOT);
+                        if (!ok) break;
+                    }
+                    if (leader) {
+                        const uint32_t bar = smem_u32(&bar_q_full[t]);
+                        mbar_arrive_expect_tx(bar, Cfg::kTileBytes);
+                        for (int x = 0; x < Cfg::kBoxes; ++x)
+                            tma_load_3d(sQ + t * Cfg::kTileBytes + x * Cfg::kBoxBytes, &tm_q, bar, x * 64,
+                                        w.q0 + t * BM, w.bh);
+                    }
+                }
+                for (int it = 0; it < 2 * w.n1 && ok; ++it, ++ring) {  // it even: K_{it/2}; odd: V_{it/2}
+                    const int slot = ring % NS, round = ring / NS;
+                    if (round > 0) {
+                        ok = wait_bar(&bar_empty[slot], (round - 1) & 1, STATUS_TIMEOUT_SLOT);
+                        if (!ok) break;
+                    }
+                    if (leader) {
+                        const uint32_t bar = smem_u32(&bar_full[slot]);
+                        const CUtensorMap *tm = (it & 1) ? &tm_v : &tm_k;
+                        if (n == 0) trace_stamp(3, it >> 1, it & 1);
+                        mbar_arrive_expect_tx(bar, Cfg::kTileBytes);
+                        for (int x = 0; x < Cfg::kBoxes; ++x)
+                            tma_load_3d(sRing + slot * Cfg::kTileBytes + x * Cfg::kBoxBytes, tm, bar, x * 64,
+                                        (it >> 1) * BN, w.bg);
+                    }
+                }
+                if (ok) id = next_tile(n, ok);
             }
             if (!ok) {
                 // abandoned: give the loads still in flight a bounded chance to land
-                for (int it = max(0, issued - NS); it < issued; ++it)
+                for (int it = max(0, ring - NS); it < ring; ++it)
                     for (uint32_t w = 0; w < WAIT_LIMIT && !mbar_try_wait(smem_u32(&bar_full[it % NS]), (it / NS) & 1); ++w) {}
             }
-        } else if (warp == 1 && lane == 0 && n1 > 0) {
+        } else if (warp == 1) {
             // =============================== MMA issuer ===============================
+            // The whole warp runs this loop so that addresses and descriptors stay
+            // warp-uniform; one elected lane issues the tcgen05 instructions.
+            const bool leader = elect_one();
             constexpr uint32_t idesc_qk = make_idesc_bf16(BM, BN, 0);
             constexpr uint32_t idesc_pv = make_idesc_bf16(BM, D, 1);
             constexpr uint64_t desc_kmajor = make_sdesc_sw128(16, 1024);
@@ -165,64 +294,104 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const uint32_t tS[2] = {tmem + Cfg::kColS0, tmem + Cfg::kColS1};
             const uint32_t tO[2] = {tmem + Cfg::kColO0, tmem + Cfg::kColO1};
             bool ok = true;
+            int ring = 0;             // ring position of the current tile's K_0
+            uint32_t np[2] = {0, 0};  // P_t hand-offs taken so far (phase of bar_p[t])
 
-            auto wait_full = [&](int idx) {
-                return mbar_wait_bounded(smem_u32(&bar_full[idx % NS]), (idx / NS) & 1, &abort_flag, STATUS_TIMEOUT_LOAD);
-            };
+            auto wait_full = [&](int idx) { return wait_bar(&bar_full[idx % NS], (idx / NS) & 1, STATUS_TIMEOUT_LOAD); };
             auto slot_addr = [&](int idx) { return sRing + (idx % NS) * Cfg::kTileBytes; };
+            // Descriptors as (low, high) words: the high word is constant per operand kind, the low
+            // word is the constant part plus address/16, so stepping along K is one 32-bit add.
+            constexpr uint32_t hi_k = uint32_t(desc_kmajor >> 32), lo_k = uint32_t(desc_kmajor);
+            constexpr uint32_t hi_v = uint32_t(desc_v >> 32), lo_v = uint32_t(desc_v);
+            const uint32_t q_lo[2] = {lo_k | (sQ >> 4), lo_k | ((sQ + Cfg::kTileBytes) >> 4)};
             auto issue_qk = [&](int t, uint32_t k_addr) {
+                if (leader) {
+                    const uint32_t k_lo = lo_k | (k_addr >> 4);
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t koff = (kk / 4) * Cfg::kBoxBytes + (kk % 4) * 32;
-                    umma_ss(tS[t], sdesc_at(desc_kmajor, sQ + t * Cfg::kTileBytes + koff),
-                            sdesc_at(desc_kmajor, k_addr + koff), idesc_qk, kk > 0);
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t koff = ((kk / 4) * Cfg::kBoxBytes + (kk % 4) * 32) >> 4;
+                        umma_ss_words(tS[t], q_lo[t] + koff, hi_k, k_lo + koff, hi_k, idesc_qk, kk > 0);
+                    }
+                    umma_commit(smem_u32(&bar_s[t]));
                 }
-                umma_commit(smem_u32(&bar_s[t]));
             };
             auto issue_pv = [&](int t, uint32_t v_addr, bool first) {
+                if (leader) {
+                    const uint32_t v_lo = lo_v | (v_addr >> 4);
 #pragma unroll
-                for (int kk = 0; kk < BN / 16; ++kk)
-                    umma_ts(tO[t], tS[t] + kk * 8, sdesc_at(desc_v, v_addr + kk * 16 * 128), idesc_pv,
-                            (!first || kk > 0));
+                    for (int kk = 0; kk < BN / 16; ++kk)
+                        umma_ts_words(tO[t], tS[t] + kk * 8, v_lo + ((kk * 16 * 128) >> 4), hi_v, idesc_pv,
+                                      (!first || kk > 0));
+                }
             };
 
-            ok = mbar_wait_bounded(smem_u32(&bar_q[0]), 0, &abort_flag, STATUS_TIMEOUT_LOAD) &&
-                 mbar_wait_bounded(smem_u32(&bar_q[1]), 0, &abort_flag, STATUS_TIMEOUT_LOAD) && wait_full(0);
-            if (ok) {
-                tc_fence_after();
-                if (n0 > 0) issue_qk(0, slot_addr(0));
-                issue_qk(1, slot_addr(0));
-                umma_commit(smem_u32(&bar_empty[0]));
-            }
-            for (int j = 0; j < n1 && ok; ++j) {
-                const int iv = 2 * j + 1, ik = 2 * j + 2;  // ring indices of V_j and K_{j+1}
-                if (j < n0) {
-                    ok = mbar_wait_bounded(smem_u32(&bar_p[0]), j & 1, &abort_flag, STATUS_TIMEOUT_SOFTMAX) && wait_full(iv);
+            int id = blockIdx.x;
+            for (int n = 0; id >= 0 && ok; ++n) {
+                const WorkTile w = decode_tile<CAUSAL>(id, p);
+                const int n0 = w.n0, n1 = w.n1;
+                if (lane == 0) trace_stamp(3, n, 7);  // start of this CTA's n-th tile
+                ok = wait_bar(&bar_q_full[0], n & 1, STATUS_TIMEOUT_LOAD) &&
+                     wait_bar(&bar_q_full[1], n & 1, STATUS_TIMEOUT_LOAD);
+                if (!ok) break;
+                if (n1 > 0) {
+                    ok = wait_full(ring);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_pv(0, slot_addr(iv), j == 0);
-                    if (j == n0 - 1) umma_commit(smem_u32(&bar_o[0]));
-                    if (j + 1 < n0) {
-                        ok = wait_full(ik);
-                        if (!ok) break;
-                        issue_qk(0, slot_addr(ik));
+                    if (n0 > 0) issue_qk(0, slot_addr(ring));
+                    issue_qk(1, slot_addr(ring));
+                    if (leader) umma_commit(smem_u32(&bar_empty[ring % NS]));
+                }
+                // Q_t is released after the last Q_t K^T of the tile (here if there is at most one)
+                if (leader && n0 <= 1) umma_commit(smem_u32(&bar_q_empty[0]));
+                if (leader && n1 <= 1) umma_commit(smem_u32(&bar_q_empty[1]));
+                for (int j = 0; j < n1 && ok; ++j) {
+                    const int iv = ring + 2 * j + 1, ik = ring + 2 * j + 2;  // ring positions of V_j and K_{j+1}
+                    if (n == 0 && lane == 0) trace_stamp(0, j, 0);
+                    // Everything this step needs from the ring and from the previous tile is checked
+                    // first, while the softmax of this step is still running; after that only the two
+                    // P hand-offs stand between this warp and the tensor pipe.
+                    ok = wait_full(iv);
+                    if (ok && j + 1 < n1) ok = wait_full(ik);
+                    if (ok && j == 0 && n > 0) {  // the previous tile's epilogue must have read O_t out of TMEM
+                        if (n0 > 0) ok = wait_bar(&bar_o_free[0], (n - 1) & 1, STATUS_TIMEOUT_SOFTMAX);
+                        ok = ok && wait_bar(&bar_o_free[1], (n - 1) & 1, STATUS_TIMEOUT_SOFTMAX);
                     }
-                }
-                ok = mbar_wait_bounded(smem_u32(&bar_p[1]), j & 1, &abort_flag, STATUS_TIMEOUT_SOFTMAX) && wait_full(iv);
-                if (!ok) break;
-                tc_fence_after();
-                issue_pv(1, slot_addr(iv), j == 0);
-                umma_commit(smem_u32(&bar_empty[iv % NS]));
-                if (j == n1 - 1) umma_commit(smem_u32(&bar_o[1]));
-                if (j + 1 < n1) {
-                    ok = wait_full(ik);
                     if (!ok) break;
-                    issue_qk(1, slot_addr(ik));
-                    umma_commit(smem_u32(&bar_empty[ik % NS]));
+                    const uint32_t v_addr = slot_addr(iv), k_addr = slot_addr(ik);
+                    if (j < n0) {
+                        ok = spin_bar(&bar_p[0], np[0] & 1, STATUS_TIMEOUT_SOFTMAX);
+                        if (!ok) break;
+                        ++np[0];
+                        if (n == 0 && lane == 0) trace_stamp(0, j, 1);
+                        tc_fence_after();
+                        issue_pv(0, v_addr, j == 0);
+                        if (leader && j == n0 - 1) umma_commit(smem_u32(&bar_o[0]));
+                        if (j + 1 < n0) {
+                            issue_qk(0, k_addr);
+                            if (leader && j + 2 == n0) umma_commit(smem_u32(&bar_q_empty[0]));
+                        }
+                    }
+                    if (n == 0 && lane == 0) trace_stamp(0, j, 2);
+                    ok = spin_bar(&bar_p[1], np[1] & 1, STATUS_TIMEOUT_SOFTMAX);
+                    if (!ok) break;
+                    ++np[1];
+                    if (n == 0 && lane == 0) trace_stamp(0, j, 3);
+                    tc_fence_after();
+                    issue_pv(1, v_addr, j == 0);
+                    if (leader) umma_commit(smem_u32(&bar_empty[iv % NS]));
+                    if (leader && j == n1 - 1) umma_commit(smem_u32(&bar_o[1]));
+                    if (j + 1 < n1) {
+                        issue_qk(1, k_addr);
+                        if (leader) umma_commit(smem_u32(&bar_empty[ik % NS]));
+                        if (leader && j + 2 == n1) umma_commit(smem_u32(&bar_q_empty[1]));
+                    }
+                    if (n == 0 && lane == 0) trace_stamp(0, j, 4);
                 }
+                ring += 2 * n1;
+                if (ok) id = next_tile(n, ok);
             }
             if (!ok) {  // abandoned: let the MMAs already issued finish before TMEM is released
-                umma_commit(smem_u32(&bar_drain));
+                if (leader) umma_commit(smem_u32(&bar_drain));
                 for (uint32_t w = 0; w < WAIT_LIMIT && !mbar_try_wait(smem_u32(&bar_drain), 0); ++w) {}
             }
         }
@@ -230,155 +399,194 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         // =============================== softmax warpgroups ===============================
         setmaxnreg_inc<Cfg::kRegsSoftmax>();
         const int t = (warp - 4) >> 2;                // sub-tile
-        const int r = tid - 128 - t * 128;            // row within the sub-tile = TMEM lane
-        const int i0 = q0 + t * BM;
-        const int i = i0 + r;                         // query row
-        const int n_t = t ? n1 : n0;
+        const int wq = warp & 3;                      // TMEM lane quadrant of this warp
+        const int r = wq * 32 + lane;                 // row within the sub-tile = TMEM lane
         const int off = p.Sk - p.Sq;
-        const uint32_t lane_sel = uint32_t((warp & 3) * 32) << 16;
+        const uint32_t lane_sel = uint32_t(wq * 32) << 16;
         const uint32_t tS = tmem + (t ? Cfg::kColS1 : Cfg::kColS0) + lane_sel;
         const uint32_t tO = tmem + (t ? Cfg::kColO1 : Cfg::kColO0) + lane_sel;
-        const uint32_t sO = sQ + t * Cfg::kTileBytes;  // O staging reuses this sub-tile's Q buffer
+        const uint32_t sO = sStage + t * Cfg::kStageOBytes + wq * (Cfg::kOutBoxRows * 128);  // this warp's 32 rows
         const float sl2 = p.scale_log2;
         const bool neg = sl2 < 0.f;
+        const bool tracer = (r == 0);
+        uint32_t ns = 0;             // S_t tiles consumed so far (phase of bar_s[t])
+        uint32_t n_out = 0;          // finished O_t accumulators taken so far (phase of bar_o[t])
+        bool ok = true;
+        bool store_pending = false;  // (lane 0) a TMA store may still be reading this warp's staging rows
 
-        if (n_t == 0) {
-            // no key visible to any row of this sub-tile: O = 0, LSE = -inf
-            if (i < p.Sq) {
-                __nv_bfloat16 *o_row = reinterpret_cast<__nv_bfloat16 *>(p.o) + (size_t(bh) * p.Sq + i) * D;
-                const uint4 z = make_uint4(0, 0, 0, 0);
-                for (int c = 0; c < D / 8; ++c) reinterpret_cast<uint4 *>(o_row)[c] = z;
-                p.lse[size_t(bh) * p.Sq + i] = -INFINITY;
-            }
-        } else {
-            float m_run = -INFINITY, l_run = 0.f;
-            bool ok = true;
-            for (int j = 0; j < n_t; ++j) {
-                ok = mbar_wait_bounded(smem_u32(&bar_s[t]), j & 1, &abort_flag, STATUS_TIMEOUT_MMA);
-                ok = __all_sync(0xffffffffu, ok);  // keep the warp together for the .sync.aligned TMEM ops
-                if (!ok) break;
-                tc_fence_after();
-                uint32_t sraw[4][32];
-#pragma unroll
-                for (int c = 0; c < 4; ++c) tmem_ld_x32(tS + c * 32, sraw[c]);
-                tmem_wait_ld();
+        int id = blockIdx.x;
+        for (int n = 0; id >= 0 && ok; ++n) {
+            const WorkTile w = decode_tile<CAUSAL>(id, p);
+            const int bh = w.bh;
+            const int i0 = w.q0 + t * BM;
+            const int i = i0 + r;                     // query row
+            const int n_t = t ? w.n1 : w.n0;
 
-                const int j0 = j * BN;
-                int lim = p.Sk - 1 - j0;  // columns c <= lim of this tile are visible to row i
-                if (CAUSAL) lim = min(lim, i + off - j0);
-                const bool need_mask = (j0 + BN > p.Sk) || (CAUSAL && (j0 + BN - 1 > i0 + off));
-
-                // ---- row extreme of the raw scores (maximum of scale*s is at max s, or min s if scale < 0)
-                float ext;
-                if (!need_mask && !neg) {
-                    float e0 = -INFINITY, e1 = -INFINITY, e2 = -INFINITY, e3 = -INFINITY;
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        e0 = fmaxf(e0, __uint_as_float(sraw[0][c]));
-                        e1 = fmaxf(e1, __uint_as_float(sraw[1][c]));
-                        e2 = fmaxf(e2, __uint_as_float(sraw[2][c]));
-                        e3 = fmaxf(e3, __uint_as_float(sraw[3][c]));
-                    }
-                    ext = fmaxf(fmaxf(e0, e1), fmaxf(e2, e3));
-                } else {
-                    ext = neg ? INFINITY : -INFINITY;
-#pragma unroll
-                    for (int c = 0; c < 128; ++c) {
-                        const float s = __uint_as_float(sraw[c >> 5][c & 31]);
-                        const bool vis = !need_mask || (c <= lim);
-                        if (neg) ext = vis ? fminf(ext, s) : ext;
-                        else     ext = vis ? fmaxf(ext, s) : ext;
-                    }
+            if (n_t == 0) {
+                // no key visible to any row of this sub-tile: O = 0, LSE = -inf
+                if (i < p.Sq) {
+                    __nv_bfloat16 *o_row = reinterpret_cast<__nv_bfloat16 *>(p.o) + (size_t(bh) * p.Sq + i) * D;
+                    const uint4 z = make_uint4(0, 0, 0, 0);
+                    for (int c = 0; c < D / 8; ++c) reinterpret_cast<uint4 *>(o_row)[c] = z;
+                    p.lse[size_t(bh) * p.Sq + i] = -INFINITY;
                 }
-                const float m_tile = (fabsf(ext) == INFINITY) ? -INFINITY : ext * sl2;
-
-                // ---- running maximum, moved lazily
-                float alpha = 1.f;
-                if (j == 0) {
-                    m_run = m_tile;
-                } else if (m_tile - m_run > kRescaleThreshold) {  // also true when m_run = -inf < m_tile
-                    const float m_use = m_tile;                   // finite here
-                    alpha = ex2_approx(m_run - m_use);
-                    m_run = m_use;
-                }
-                if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-                    // O <- alpha * O.  S_t(j) ready implies P_t V_{j-1} has finished (in-order tensor pipe).
-#pragma unroll
-                    for (int c = 0; c < D / 32; ++c) {
-                        uint32_t oc[32];
-                        tmem_ld_x32(tO + c * 32, oc);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) oc[e] = __float_as_uint(__uint_as_float(oc[e]) * alpha);
-                        tmem_st_x32(tO + c * 32, oc);
-                    }
-                }
-                const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
-
-                // ---- p = exp2(scale*log2e*s - m); row sum in fp32; P -> bf16 pairs into TMEM
-                float sum0 = 0.f, sum1 = 0.f;
-#pragma unroll
-                for (int cc = 0; cc < 4; ++cc) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int e = 0; e < 32; e += 2) {
-                        float p0 = ex2_approx(fmaf(__uint_as_float(sraw[cc][e]), sl2, neg_m));
-                        float p1 = ex2_approx(fmaf(__uint_as_float(sraw[cc][e + 1]), sl2, neg_m));
-                        if (need_mask) {
-                            p0 = (cc * 32 + e <= lim) ? p0 : 0.f;
-                            p1 = (cc * 32 + e + 1 <= lim) ? p1 : 0.f;
-                        }
-                        sum0 += p0;
-                        sum1 += p1;
-                        pk[e >> 1] = pack_bf16x2(p0, p1);
-                    }
-                    tmem_st_x16(tS + cc * 16, pk);
-                }
-                l_run = l_run * alpha + (sum0 + sum1);
-
-                tmem_wait_st();
-                tc_fence_before();
+                // O_t was not used: hand it back at once so its barrier completes once per tile
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&bar_p[t]));
-            }
-
-            // ---- epilogue: O / l -> bf16 -> shared (TMA layout) -> global; LSE = ln2 * (m + log2 l)
-            if (ok) ok = mbar_wait_bounded(smem_u32(&bar_o[t]), 0, &abort_flag, STATUS_TIMEOUT_MMA);
-            ok = __all_sync(0xffffffffu, ok);
-            if (ok) {
-                tc_fence_after();
-                const float inv_l = (l_run > 0.f) ? 1.f / l_run : 0.f;
+                if (lane == 0) mbar_arrive(smem_u32(&bar_o_free[t]));
+            } else {
+                float m_run = -INFINITY, l_run = 0.f;
+                for (int j = 0; j < n_t; ++j) {
+                    if (n == 0 && tracer) trace_stamp(1 + t, j, 0);
+                    ok = wait_bar(&bar_s[t], ns & 1, STATUS_TIMEOUT_MMA);
+                    if (!ok) break;
+                    ++ns;
+                    if (n == 0 && tracer) trace_stamp(1 + t, j, 1);
+                    tc_fence_after();
+                    uint32_t sraw[4][32];
 #pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t oc[32];
-                    tmem_ld_x32(tO + c * 32, oc);
+                    for (int c = 0; c < 4; ++c) tmem_ld_x32(tS + c * 32, sraw[c]);
                     tmem_wait_ld();
+                    if (n == 0 && tracer) trace_stamp(1 + t, j, 2);
+
+                    const int j0 = j * BN;
+                    int lim = p.Sk - 1 - j0;  // columns c <= lim of this tile are visible to row i
+                    if (CAUSAL) lim = min(lim, i + off - j0);
+                    const bool need_mask = (j0 + BN > p.Sk) || (CAUSAL && (j0 + BN - 1 > i0 + off));
+
+                    // ---- row extreme of the raw scores (maximum of scale*s is at max s, or min s if scale < 0)
+                    float ext;
+                    if (!need_mask && !neg) {
+                        float e0 = -INFINITY, e1 = -INFINITY, e2 = -INFINITY, e3 = -INFINITY;
 #pragma unroll
-                    for (int e = 0; e < 32; e += 8) {
-                        uint4 w;
-                        w.x = pack_bf16x2(__uint_as_float(oc[e + 0]) * inv_l, __uint_as_float(oc[e + 1]) * inv_l);
-                        w.y = pack_bf16x2(__uint_as_float(oc[e + 2]) * inv_l, __uint_as_float(oc[e + 3]) * inv_l);
-                        w.z = pack_bf16x2(__uint_as_float(oc[e + 4]) * inv_l, __uint_as_float(oc[e + 5]) * inv_l);
-                        w.w = pack_bf16x2(__uint_as_float(oc[e + 6]) * inv_l, __uint_as_float(oc[e + 7]) * inv_l);
-                        // 16-byte chunk `ch` of row r, in the 128-byte-swizzled box layout TMA expects
-                        const int ch = (c * 32 + e) >> 3;
-                        const uint32_t addr = sO + (ch >> 3) * Cfg::kBoxBytes + r * 128 + (((ch & 7) ^ (r & 7)) << 4);
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w.x), "r"(w.y),
-                                     "r"(w.z), "r"(w.w) : "memory");
+                        for (int c = 0; c < 32; c += 2) {
+                            e0 = max3(e0, __uint_as_float(sraw[0][c]), __uint_as_float(sraw[0][c + 1]));
+                            e1 = max3(e1, __uint_as_float(sraw[1][c]), __uint_as_float(sraw[1][c + 1]));
+                            e2 = max3(e2, __uint_as_float(sraw[2][c]), __uint_as_float(sraw[2][c + 1]));
+                            e3 = max3(e3, __uint_as_float(sraw[3][c]), __uint_as_float(sraw[3][c + 1]));
+                        }
+                        ext = fmaxf(fmaxf(e0, e1), fmaxf(e2, e3));
+                    } else {
+                        ext = neg ? INFINITY : -INFINITY;
+#pragma unroll
+                        for (int c = 0; c < 128; ++c) {
+                            const float s = __uint_as_float(sraw[c >> 5][c & 31]);
+                            const bool vis = !need_mask || (c <= lim);
+                            if (neg) ext = vis ? fminf(ext, s) : ext;
+                            else     ext = vis ? fmaxf(ext, s) : ext;
+                        }
+                    }
+                    const float m_tile = (fabsf(ext) == INFINITY) ? -INFINITY : ext * sl2;
+
+                    // ---- running maximum, moved lazily
+                    float alpha = 1.f;
+                    if (j == 0) {
+                        m_run = m_tile;
+                    } else if (m_tile - m_run > kRescaleThreshold) {  // also true when m_run = -inf < m_tile
+                        alpha = ex2_approx(m_run - m_tile);           // m_tile is finite here
+                        m_run = m_tile;
+                    }
+                    if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+                        // O <- alpha * O.  S_t(j) ready implies P_t V_{j-1} has finished (in-order tensor pipe).
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t oc[32];
+                            tmem_ld_x32(tO + c * 32, oc);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) oc[e] = __float_as_uint(__uint_as_float(oc[e]) * alpha);
+                            tmem_st_x32(tO + c * 32, oc);
+                        }
+                    }
+                    const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
+                    if (n == 0 && tracer) trace_stamp(1 + t, j, 3);
+
+                    // ---- p = exp2(scale*log2e*s - m); row sum in fp32; P -> bf16 pairs into TMEM
+                    float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+                    const float2 sc2 = make_float2(sl2, sl2), nm2 = make_float2(neg_m, neg_m);
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) {
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int e = 0; e < 32; e += 2) {
+                            const float2 x = __ffma2_rn(
+                                make_float2(__uint_as_float(sraw[cc][e]), __uint_as_float(sraw[cc][e + 1])), sc2, nm2);
+                            float2 pr;
+                            if ((kFmaPipeExpMask >> ((e >> 1) & 7)) & 1) {
+                                pr = exp2_fma_pipe(x);
+                            } else {
+                                pr.x = ex2_approx(x.x);
+                                pr.y = ex2_approx(x.y);
+                            }
+                            if (need_mask) {
+                                pr.x = (cc * 32 + e <= lim) ? pr.x : 0.f;
+                                pr.y = (cc * 32 + e + 1 <= lim) ? pr.y : 0.f;
+                            }
+                            if (e & 2) acc1 = __fadd2_rn(acc1, pr);  // fp32 probabilities, before rounding to bf16
+                            else       acc0 = __fadd2_rn(acc0, pr);
+                            pk[e >> 1] = pack_bf16x2(pr.x, pr.y);
+                        }
+                        tmem_st_x16(tS + cc * 16, pk);
+                    }
+                    l_run = l_run * alpha + ((acc0.x + acc0.y) + (acc1.x + acc1.y));
+                    if (n == 0 && tracer) trace_stamp(1 + t, j, 4);
+
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bar_p[t]));
+                    if (n == 0 && tracer) trace_stamp(1 + t, j, 5);
+                }
+
+                // ---- epilogue: O / l -> bf16 -> shared (TMA layout) -> global; LSE = ln2 * (m + log2 l)
+                if (ok) ok = wait_bar(&bar_o[t], n_out & 1, STATUS_TIMEOUT_MMA);
+                if (ok) {
+                    ++n_out;
+                    tc_fence_after();
+                    const float inv_l = (l_run > 0.f) ? 1.f / l_run : 0.f;
+                    if (i < p.Sq)
+                        p.lse[size_t(bh) * p.Sq + i] =
+                            (l_run > 0.f) ? (m_run + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+#pragma unroll
+                    for (int x = 0; x < Cfg::kBoxes; ++x) {  // 64 columns of O at a time through the staging rows
+                        uint32_t oc[2][32];
+                        tmem_ld_x32(tO + x * 64, oc[0]);
+                        tmem_ld_x32(tO + x * 64 + 32, oc[1]);
+                        tmem_wait_ld();
+                        if (x == Cfg::kBoxes - 1) {  // O_t is in registers: the next tile may overwrite it
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(smem_u32(&bar_o_free[t]));
+                        }
+                        // this warp's previous TMA store must have finished reading the staging rows
+                        if (lane == 0 && store_pending) tma_store_wait_read();
+                        __syncwarp();
+#pragma unroll
+                        for (int e = 0; e < 64; e += 8) {
+                            const uint32_t *src = &oc[e >> 5][e & 31];
+                            uint4 v4;
+                            v4.x = pack_bf16x2(__uint_as_float(src[0]) * inv_l, __uint_as_float(src[1]) * inv_l);
+                            v4.y = pack_bf16x2(__uint_as_float(src[2]) * inv_l, __uint_as_float(src[3]) * inv_l);
+                            v4.z = pack_bf16x2(__uint_as_float(src[4]) * inv_l, __uint_as_float(src[5]) * inv_l);
+                            v4.w = pack_bf16x2(__uint_as_float(src[6]) * inv_l, __uint_as_float(src[7]) * inv_l);
+                            // 16-byte chunk `ch` of row `lane`, in the 128-byte-swizzled layout TMA expects
+                            const int ch = e >> 3;
+                            const uint32_t addr = sO + lane * 128 + ((ch ^ (lane & 7)) << 4);
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v4.x), "r"(v4.y),
+                                         "r"(v4.z), "r"(v4.w) : "memory");
+                        }
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0 && i0 + wq * 32 < p.Sq) {
+                            tma_store_3d(&tm_o, sO, x * 64, i0 + wq * 32, bh);
+                            tma_store_commit();
+                            store_pending = true;
+                        }
                     }
                 }
-                if (i < p.Sq)
-                    p.lse[size_t(bh) * p.Sq + i] =
-                        (l_run > 0.f) ? (m_run + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
-                fence_proxy_async_smem();
             }
-            named_barrier_sync(1 + t, 128);  // reached by every thread of the warpgroup, abandoned or not
-            if (r == 0 && i0 < p.Sq && abort_flag == 0) {
-                for (int x = 0; x < Cfg::kBoxes; ++x) tma_store_3d(&tm_o, sO + x * Cfg::kBoxBytes, x * 64, i0, bh);
-                tma_store_commit();
-                tma_store_wait_all();
-            }
+            if (ok) id = next_tile(n, ok);
         }
+        if (lane == 0 && store_pending) tma_store_wait_all();
     }
 
     // ---- common exit: every thread arrives, then TMEM is released

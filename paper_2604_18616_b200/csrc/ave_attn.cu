@@ -144,7 +144,7 @@ int ave_attn_fwd(const void *q, const void *k, const void *v, void *o, float *ls
 
     CUtensorMap tq, tk, tv, to;
     if (!encode_map(&tq, q, D, Sq, (long long)B * H, ave::BM)) return AVE_ERR_CUDA;
-    if (!encode_map(&to, o, D, Sq, (long long)B * H, ave::BM)) return AVE_ERR_CUDA;
+    if (!encode_map(&to, o, D, Sq, (long long)B * H, ave::WsCfg<128>::kOutBoxRows)) return AVE_ERR_CUDA;
     if (!encode_map(&tk, k, D, Sk, (long long)B * Hkv, ave::BN)) return AVE_ERR_CUDA;
     if (!encode_map(&tv, v, D, Sk, (long long)B * Hkv, ave::BN)) return AVE_ERR_CUDA;
 
@@ -155,8 +155,21 @@ int ave_attn_fwd(const void *q, const void *k, const void *v, void *o, float *ls
     p.Hkv = Hkv;
     p.Sq = Sq;
     p.Sk = Sk;
+    p.BH = B * H;
     p.n_qblk = (Sq + 2 * ave::BM - 1) / (2 * ave::BM);
-    p.total_blocks = p.n_qblk * B * H;
+    p.total_blocks = p.n_qblk * p.BH;
+    {
+        // Launch (b, h) pairs in groups whose K and V together stay within a slice of L2,
+        // whole key/value heads at a time.
+        const long long kv_bytes_per_kv_head = 2ll * Sk * D * 2;
+        const int G = H / Hkv;
+        const long long budget = 24ll << 20;
+        long long kv_heads = budget / kv_bytes_per_kv_head;
+        if (kv_heads < 1) kv_heads = 1;
+        long long hpg = kv_heads * G;
+        if (hpg > p.BH) hpg = p.BH;
+        p.heads_per_group = int(hpg);
+    }
     p.scale_log2 = scale * 1.4426950408889634f;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -249,6 +262,16 @@ const char *ave_attn_strerror(int status) {
 }
 
 int ave_attn_version(void) { return kVersion; }
+
+#ifdef AVE_TRACE
+// Trace builds only (not part of the public interface): copies the role
+// timeline of the traced CTA, TRACE_ROLES x TRACE_ITERS x TRACE_SLOTS clocks.
+int ave_attn_trace_read(long long *out) {
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpyFromSymbol(out, ave::g_trace, sizeof(ave::g_trace));
+    return e == cudaSuccess ? AVE_OK : AVE_ERR_CUDA;
+}
+#endif
 
 int ave_attn_last_cuda_error(void) { return t_last_cuda_error; }
 
