@@ -22,9 +22,11 @@ constexpr unsigned int STATUS_TIMEOUT_MMA = 2u;      // waiting for a tcgen05.co
 constexpr unsigned int STATUS_TIMEOUT_SOFTMAX = 4u;  // MMA warp waiting for P
 constexpr unsigned int STATUS_TIMEOUT_SLOT = 8u;     // producer waiting for a free stage
 
-// Upper bound on mbarrier polls before a wait is abandoned (a fraction of a
-// second; legitimate waits last microseconds).
-constexpr uint32_t WAIT_LIMIT = 1u << 21;
+// A wait is abandoned after this many SM clock cycles (a fraction of a second;
+// legitimate waits last microseconds).
+constexpr long long WAIT_LIMIT_CYCLES = 1ll << 29;
+// Poll limit of the short non-suspending drain loops that run after a wait was abandoned.
+constexpr uint32_t WAIT_LIMIT = 1u << 16;
 
 struct FwdParams {
     void *o;          // bf16 [B, H, Sq, D]
@@ -76,14 +78,19 @@ __device__ __forceinline__ void trace_stamp(int role, int iter, int slot) {
 __device__ __forceinline__ void trace_stamp(int, int, int) {}
 #endif
 
-// Poll an mbarrier phase with an iteration limit.  Returns false when the
-// limit was reached or another thread of the CTA has already given up;
-// `abort_flag` is a shared-memory word all roles watch.
+// Wait for an mbarrier phase, for a bounded TIME (one mbarrier.try_wait may
+// itself suspend the thread for a hardware-chosen while, so counting polls
+// does not bound the wait).  Returns false when the time ran out or another
+// thread of the CTA has already given up; `abort_flag` is a shared-memory
+// word all roles watch.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int *abort_flag,
                                                   unsigned int code) {
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 0x3FFu) == 0x3FFu && *abort_flag != 0) return false;
+        if (*abort_flag != 0) return false;
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
     }
     *abort_flag = 1;
     atomicOr(&g_device_status, code);
@@ -93,12 +100,14 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
 // The same with a non-suspending poll: the waiter notices the completion within a
 // few tens of cycles instead of after a wake-up, at the price of issue slots.
 // For the one warp whose reaction time is on the critical path.
-constexpr uint32_t SPIN_LIMIT = 1u << 25;
 __device__ __forceinline__ bool mbar_spin_bounded(uint32_t bar, uint32_t parity, volatile int *abort_flag,
                                                   unsigned int code) {
-    for (uint32_t it = 0; it < SPIN_LIMIT; ++it) {
+    for (uint32_t it = 0;; ++it) {
         if (mbar_test_wait(bar, parity)) return true;
-        if ((it & 0xFFFFu) == 0xFFFFu && *abort_flag != 0) return false;
+        if ((it & 0x3FFu) == 0x3FFu) {
+            if (*abort_flag != 0) return false;
+            if (it >= (1u << 24)) break;  // 2^24 polls of a few tens of cycles each
+        }
     }
     *abort_flag = 1;
     atomicOr(&g_device_status, code);

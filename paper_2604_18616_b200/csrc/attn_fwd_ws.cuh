@@ -42,7 +42,12 @@ struct WsCfg {
     static constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO0 = 256, kColO1 = 384;
     static constexpr int kRegsLight = 64;                    // producer / MMA / scheduler warpgroup
     static constexpr int kRegsSoftmax = 216;                 // softmax warpgroups
-    static constexpr int kTileConsumers = 10;                // producer + MMA + 8 softmax warps read each tile id
+    // setmaxnreg only moves registers inside what the CTA was given at launch (kThreads x the
+    // per-thread count ptxas reports, 168 for 384 threads); asking for more blocks forever.
+    static constexpr int kRegsAtLaunch = 168;
+    static_assert(128 * kRegsLight + 256 * kRegsSoftmax <= kThreads * kRegsAtLaunch,
+                  "register split exceeds the CTA's allocation");
+    static constexpr int kTileConsumers = 10;               // producer + MMA + 8 softmax warps read each tile id
 };
 
 // Rescale O only when the running maximum moved by more than this many
@@ -57,6 +62,12 @@ constexpr float kRescaleThreshold = 8.0f;
 #define AVE_FMA_EXP_MASK 0x00
 #endif
 constexpr unsigned kFmaPipeExpMask = AVE_FMA_EXP_MASK;
+
+// Trace builds record the role timeline of this one of a CTA's tiles (0 = its first).
+#ifndef AVE_TRACE_TILE
+#define AVE_TRACE_TILE 0
+#endif
+constexpr int kTraceTile = AVE_TRACE_TILE;
 
 template <int N>
 __device__ __forceinline__ void setmaxnreg_inc() {
@@ -268,7 +279,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     if (leader) {
                         const uint32_t bar = smem_u32(&bar_full[slot]);
                         const CUtensorMap *tm = (it & 1) ? &tm_v : &tm_k;
-                        if (n == 0) trace_stamp(3, it >> 1, it & 1);
+                        if (n == kTraceTile) trace_stamp(3, it >> 1, it & 1);
                         mbar_arrive_expect_tx(bar, Cfg::kTileBytes);
                         for (int x = 0; x < Cfg::kBoxes; ++x)
                             tma_load_3d(sRing + slot * Cfg::kTileBytes + x * Cfg::kBoxBytes, tm, bar, x * 64,
@@ -280,7 +291,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             if (!ok) {
                 // abandoned: give the loads still in flight a bounded chance to land
                 for (int it = max(0, ring - NS); it < ring; ++it)
-                    for (uint32_t w = 0; w < WAIT_LIMIT && !mbar_try_wait(smem_u32(&bar_full[it % NS]), (it / NS) & 1); ++w) {}
+                    for (uint32_t w = 0; w < WAIT_LIMIT && !mbar_test_wait(smem_u32(&bar_full[it % NS]), (it / NS) & 1); ++w) {}
             }
         } else if (warp == 1) {
             // =============================== MMA issuer ===============================
@@ -346,7 +357,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 if (leader && n1 <= 1) umma_commit(smem_u32(&bar_q_empty[1]));
                 for (int j = 0; j < n1 && ok; ++j) {
                     const int iv = ring + 2 * j + 1, ik = ring + 2 * j + 2;  // ring positions of V_j and K_{j+1}
-                    if (n == 0 && lane == 0) trace_stamp(0, j, 0);
+                    if (n == kTraceTile && lane == 0) trace_stamp(0, j, 0);
                     // Everything this step needs from the ring and from the previous tile is checked
                     // first, while the softmax of this step is still running; after that only the two
                     // P hand-offs stand between this warp and the tensor pipe.
@@ -362,7 +373,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         ok = spin_bar(&bar_p[0], np[0] & 1, STATUS_TIMEOUT_SOFTMAX);
                         if (!ok) break;
                         ++np[0];
-                        if (n == 0 && lane == 0) trace_stamp(0, j, 1);
+                        if (n == kTraceTile && lane == 0) trace_stamp(0, j, 1);
                         tc_fence_after();
                         issue_pv(0, v_addr, j == 0);
                         if (leader && j == n0 - 1) umma_commit(smem_u32(&bar_o[0]));
@@ -371,11 +382,11 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                             if (leader && j + 2 == n0) umma_commit(smem_u32(&bar_q_empty[0]));
                         }
                     }
-                    if (n == 0 && lane == 0) trace_stamp(0, j, 2);
+                    if (n == kTraceTile && lane == 0) trace_stamp(0, j, 2);
                     ok = spin_bar(&bar_p[1], np[1] & 1, STATUS_TIMEOUT_SOFTMAX);
                     if (!ok) break;
                     ++np[1];
-                    if (n == 0 && lane == 0) trace_stamp(0, j, 3);
+                    if (n == kTraceTile && lane == 0) trace_stamp(0, j, 3);
                     tc_fence_after();
                     issue_pv(1, v_addr, j == 0);
                     if (leader) umma_commit(smem_u32(&bar_empty[iv % NS]));
@@ -385,14 +396,14 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         if (leader) umma_commit(smem_u32(&bar_empty[ik % NS]));
                         if (leader && j + 2 == n1) umma_commit(smem_u32(&bar_q_empty[1]));
                     }
-                    if (n == 0 && lane == 0) trace_stamp(0, j, 4);
+                    if (n == kTraceTile && lane == 0) trace_stamp(0, j, 4);
                 }
                 ring += 2 * n1;
                 if (ok) id = next_tile(n, ok);
             }
             if (!ok) {  // abandoned: let the MMAs already issued finish before TMEM is released
                 if (leader) umma_commit(smem_u32(&bar_drain));
-                for (uint32_t w = 0; w < WAIT_LIMIT && !mbar_try_wait(smem_u32(&bar_drain), 0); ++w) {}
+                for (uint32_t w = 0; w < WAIT_LIMIT && !mbar_test_wait(smem_u32(&bar_drain), 0); ++w) {}
             }
         }
     } else {
@@ -436,17 +447,17 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             } else {
                 float m_run = -INFINITY, l_run = 0.f;
                 for (int j = 0; j < n_t; ++j) {
-                    if (n == 0 && tracer) trace_stamp(1 + t, j, 0);
+                    if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 0);
                     ok = wait_bar(&bar_s[t], ns & 1, STATUS_TIMEOUT_MMA);
                     if (!ok) break;
                     ++ns;
-                    if (n == 0 && tracer) trace_stamp(1 + t, j, 1);
+                    if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 1);
                     tc_fence_after();
                     uint32_t sraw[4][32];
 #pragma unroll
                     for (int c = 0; c < 4; ++c) tmem_ld_x32(tS + c * 32, sraw[c]);
                     tmem_wait_ld();
-                    if (n == 0 && tracer) trace_stamp(1 + t, j, 2);
+                    if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 2);
 
                     const int j0 = j * BN;
                     int lim = p.Sk - 1 - j0;  // columns c <= lim of this tile are visible to row i
@@ -498,7 +509,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         }
                     }
                     const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
-                    if (n == 0 && tracer) trace_stamp(1 + t, j, 3);
+                    if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 3);
 
                     // ---- p = exp2(scale*log2e*s - m); row sum in fp32; P -> bf16 pairs into TMEM
                     float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
@@ -528,13 +539,13 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         tmem_st_x16(tS + cc * 16, pk);
                     }
                     l_run = l_run * alpha + ((acc0.x + acc0.y) + (acc1.x + acc1.y));
-                    if (n == 0 && tracer) trace_stamp(1 + t, j, 4);
+                    if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 4);
 
                     tmem_wait_st();
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&bar_p[t]));
-                    if (n == 0 && tracer) trace_stamp(1 + t, j, 5);
+                    if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 5);
                 }
 
                 // ---- epilogue: O / l -> bf16 -> shared (TMA layout) -> global; LSE = ln2 * (m + log2 l)
