@@ -257,11 +257,22 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             int id = blockIdx.x;
             for (int n = 0; id >= 0 && ok; ++n) {
                 const WorkTile w = decode_tile<CAUSAL>(id, p);
-                for (int t = 0; t < 2 && ok; ++t) {
-                    if (n > 0) {  // the previous tile's last Q_t K^T has finished reading this buffer
-                        ok = wait_bar(&bar_q_empty[t], (n - 1) & 1, STATUS_TIMEOUT_SLOT);
-                        if (!ok) break;
+                // Q_t of this tile goes in as soon as the previous tile's last Q_t K^T has retired.
+                // Q_1 is released later than Q_0 (causal sub-tile 1 runs one step longer), and the
+                // first K/V tiles must not queue behind it, so a Q load that cannot go yet stays
+                // pending and is retried between the K/V loads.
+                bool q_pending[2] = {true, true};
+                auto try_load_q = [&](int t, bool blocking) {
+                    if (!q_pending[t]) return;
+                    if (n > 0) {
+                        if (blocking) {
+                            ok = wait_bar(&bar_q_empty[t], (n - 1) & 1, STATUS_TIMEOUT_SLOT);
+                            if (!ok) return;
+                        } else if (!__all_sync(0xffffffffu, mbar_test_wait(smem_u32(&bar_q_empty[t]), (n - 1) & 1))) {
+                            return;
+                        }
                     }
+                    q_pending[t] = false;
                     if (leader) {
                         const uint32_t bar = smem_u32(&bar_q_full[t]);
                         mbar_arrive_expect_tx(bar, Cfg::kTileBytes);
@@ -269,12 +280,35 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                             tma_load_3d(sQ + t * Cfg::kTileBytes + x * Cfg::kBoxBytes, &tm_q, bar, x * 64,
                                         w.q0 + t * BM, w.bh);
                     }
-                }
+                };
+                try_load_q(0, false);
+                try_load_q(1, false);
                 for (int it = 0; it < 2 * w.n1 && ok; ++it, ++ring) {  // it even: K_{it/2}; odd: V_{it/2}
                     const int slot = ring % NS, round = ring / NS;
                     if (round > 0) {
-                        ok = wait_bar(&bar_empty[slot], (round - 1) & 1, STATUS_TIMEOUT_SLOT);
+                        // Poll for the slot without blocking: a Q buffer may free up first, and the MMA
+                        // warp may be waiting for that Q before it releases any more slots.
+                        const long long t0 = clock64();
+                        for (;;) {
+                            try_load_q(0, false);
+                            try_load_q(1, false);
+                            if (__all_sync(0xffffffffu, mbar_test_wait(smem_u32(&bar_empty[slot]), (round - 1) & 1))) break;
+                            if (*reinterpret_cast<volatile int *>(&abort_flag) != 0) {
+                                ok = false;
+                                break;
+                            }
+                            if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+                                abort_flag = 1;
+                                atomicOr(&g_device_status, STATUS_TIMEOUT_SLOT);
+                                ok = false;
+                                break;
+                            }
+                            __nanosleep(40);
+                        }
                         if (!ok) break;
+                    } else {
+                        try_load_q(0, false);
+                        try_load_q(1, false);
                     }
                     if (leader) {
                         const uint32_t bar = smem_u32(&bar_full[slot]);
@@ -286,6 +320,8 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                                         (it >> 1) * BN, w.bg);
                     }
                 }
+                if (ok) try_load_q(0, true);
+                if (ok) try_load_q(1, true);
                 if (ok) id = next_tile(n, ok);
             }
             if (!ok) {
@@ -336,25 +372,41 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 }
             };
 
+            // First step of sub-tile t in tile number `tn` (tile `wt`, whose K_0 sits at ring position
+            // `ring0`): S_t = Q_t K_0^T.  Issued as soon as sub-tile t has finished the tile before, so
+            // the next tile's first scores are computed while the other sub-tile is still at work.
+            auto start_subtile = [&](int t, const WorkTile &wt, int tn, int ring0) {
+                const int n_t = t ? wt.n1 : wt.n0;
+                ok = wait_bar(&bar_q_full[t], tn & 1, STATUS_TIMEOUT_LOAD);
+                if (ok && n_t > 0) ok = wait_full(ring0);
+                if (!ok) return;
+                if (n_t > 0) {
+                    tc_fence_after();
+                    issue_qk(t, slot_addr(ring0));
+                }
+                // sub-tile 1 always visits at least as many key tiles as sub-tile 0: it is the last user of K_0
+                if (leader && t == 1 && wt.n1 > 0) umma_commit(smem_u32(&bar_empty[ring0 % NS]));
+                // Q_t is released after the last Q_t K^T of the tile (here if there is at most one)
+                if (leader && n_t <= 1) umma_commit(smem_u32(&bar_q_empty[t]));
+            };
+
             int id = blockIdx.x;
+            WorkTile w = decode_tile<CAUSAL>(id, p);
+            start_subtile(0, w, 0, 0);
+            if (ok) start_subtile(1, w, 0, 0);
             for (int n = 0; id >= 0 && ok; ++n) {
-                const WorkTile w = decode_tile<CAUSAL>(id, p);
                 const int n0 = w.n0, n1 = w.n1;
                 if (lane == 0) trace_stamp(3, n, 7);  // start of this CTA's n-th tile
-                ok = wait_bar(&bar_q_full[0], n & 1, STATUS_TIMEOUT_LOAD) &&
-                     wait_bar(&bar_q_full[1], n & 1, STATUS_TIMEOUT_LOAD);
+                // the tile after this one (its first steps are issued from inside this tile's loop)
+                const int id_next = next_tile(n, ok);
                 if (!ok) break;
-                if (n1 > 0) {
-                    ok = wait_full(ring);
-                    if (!ok) break;
-                    tc_fence_after();
-                    if (n0 > 0) issue_qk(0, slot_addr(ring));
-                    issue_qk(1, slot_addr(ring));
-                    if (leader) umma_commit(smem_u32(&bar_empty[ring % NS]));
+                WorkTile w_next = w;
+                if (id_next >= 0) w_next = decode_tile<CAUSAL>(id_next, p);
+                const int ring_next = ring + 2 * n1;
+                if (id_next >= 0 && n1 == 0) {  // nothing to do in this tile at all
+                    start_subtile(0, w_next, n + 1, ring_next);
+                    if (ok) start_subtile(1, w_next, n + 1, ring_next);
                 }
-                // Q_t is released after the last Q_t K^T of the tile (here if there is at most one)
-                if (leader && n0 <= 1) umma_commit(smem_u32(&bar_q_empty[0]));
-                if (leader && n1 <= 1) umma_commit(smem_u32(&bar_q_empty[1]));
                 for (int j = 0; j < n1 && ok; ++j) {
                     const int iv = ring + 2 * j + 1, ik = ring + 2 * j + 2;  // ring positions of V_j and K_{j+1}
                     if (n == kTraceTile && lane == 0) trace_stamp(0, j, 0);
@@ -380,6 +432,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         if (j + 1 < n0) {
                             issue_qk(0, k_addr);
                             if (leader && j + 2 == n0) umma_commit(smem_u32(&bar_q_empty[0]));
+                        } else if (id_next >= 0) {
+                            start_subtile(0, w_next, n + 1, ring_next);  // sub-tile 0 moves on to the next tile
+                            if (!ok) break;
                         }
                     }
                     if (n == kTraceTile && lane == 0) trace_stamp(0, j, 2);
@@ -395,11 +450,16 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         issue_qk(1, k_addr);
                         if (leader) umma_commit(smem_u32(&bar_empty[ik % NS]));
                         if (leader && j + 2 == n1) umma_commit(smem_u32(&bar_q_empty[1]));
+                    } else if (id_next >= 0) {
+                        if (n0 == 0) start_subtile(0, w_next, n + 1, ring_next);  // sub-tile 0 had nothing to do here
+                        if (ok) start_subtile(1, w_next, n + 1, ring_next);
+                        if (!ok) break;
                     }
                     if (n == kTraceTile && lane == 0) trace_stamp(0, j, 4);
                 }
-                ring += 2 * n1;
-                if (ok) id = next_tile(n, ok);
+                ring = ring_next;
+                id = id_next;
+                w = w_next;
             }
             if (!ok) {  // abandoned: let the MMAs already issued finish before TMEM is released
                 if (leader) umma_commit(smem_u32(&bar_drain));
@@ -465,8 +525,17 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     const bool need_mask = (j0 + BN > p.Sk) || (CAUSAL && (j0 + BN - 1 > i0 + off));
 
                     // ---- row extreme of the raw scores (maximum of scale*s is at max s, or min s if scale < 0)
+                    // With a positive scale a masked score is simply replaced by -inf: it then drops out
+                    // of the maximum and its probability exp2(-inf) is exactly 0.  Zero and negative
+                    // scales (where -inf * scale is not -inf) take the explicit, slower path below.
+                    const bool generic = !(sl2 > 0.f);
+                    if (need_mask && !generic) {
+#pragma unroll
+                        for (int c = 0; c < 128; ++c)
+                            sraw[c >> 5][c & 31] = (c <= lim) ? sraw[c >> 5][c & 31] : 0xff800000u;
+                    }
                     float ext;
-                    if (!need_mask && !neg) {
+                    if (!generic) {
                         float e0 = -INFINITY, e1 = -INFINITY, e2 = -INFINITY, e3 = -INFINITY;
 #pragma unroll
                         for (int c = 0; c < 32; c += 2) {
@@ -528,7 +597,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                                 pr.x = ex2_approx(x.x);
                                 pr.y = ex2_approx(x.y);
                             }
-                            if (need_mask) {
+                            if (need_mask && generic) {
                                 pr.x = (cc * 32 + e <= lim) ? pr.x : 0.f;
                                 pr.y = (cc * 32 + e + 1 <= lim) ? pr.y : 0.f;
                             }
