@@ -163,7 +163,7 @@ int ave_attn_fwd(const void *q, const void *k, const void *v, void *o, float *ls
         // whole key/value heads at a time.
         const long long kv_bytes_per_kv_head = 2ll * Sk * D * 2;
         const int G = H / Hkv;
-        const long long budget = 24ll << 20;
+        const long long budget = 64ll << 20;
         long long kv_heads = budget / kv_bytes_per_kv_head;
         if (kv_heads < 1) kv_heads = 1;
         long long hpg = kv_heads * G;
