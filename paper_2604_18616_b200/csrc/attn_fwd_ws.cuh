@@ -534,39 +534,65 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         for (int c = 0; c < 128; ++c)
                             sraw[c >> 5][c & 31] = (c <= lim) ? sraw[c >> 5][c & 31] : 0xff800000u;
                     }
-                    float ext;
-                    if (!generic) {
-                        float e0 = -INFINITY, e1 = -INFINITY, e2 = -INFINITY, e3 = -INFINITY;
+                    // Row extreme of the (masked) raw scores, as scale*log2(e)*s; -inf if nothing is visible.
+                    auto tile_max = [&]() -> float {
+                        float ext;
+                        if (!generic) {
+                            float e0 = -INFINITY, e1 = -INFINITY, e2 = -INFINITY, e3 = -INFINITY;
 #pragma unroll
-                        for (int c = 0; c < 32; c += 2) {
-                            e0 = max3(e0, __uint_as_float(sraw[0][c]), __uint_as_float(sraw[0][c + 1]));
-                            e1 = max3(e1, __uint_as_float(sraw[1][c]), __uint_as_float(sraw[1][c + 1]));
-                            e2 = max3(e2, __uint_as_float(sraw[2][c]), __uint_as_float(sraw[2][c + 1]));
-                            e3 = max3(e3, __uint_as_float(sraw[3][c]), __uint_as_float(sraw[3][c + 1]));
-                        }
-                        ext = fmaxf(fmaxf(e0, e1), fmaxf(e2, e3));
-                    } else {
-                        ext = neg ? INFINITY : -INFINITY;
+                            for (int c = 0; c < 32; c += 2) {
+                                e0 = max3(e0, __uint_as_float(sraw[0][c]), __uint_as_float(sraw[0][c + 1]));
+                                e1 = max3(e1, __uint_as_float(sraw[1][c]), __uint_as_float(sraw[1][c + 1]));
+                                e2 = max3(e2, __uint_as_float(sraw[2][c]), __uint_as_float(sraw[2][c + 1]));
+                                e3 = max3(e3, __uint_as_float(sraw[3][c]), __uint_as_float(sraw[3][c + 1]));
+                            }
+                            ext = fmaxf(fmaxf(e0, e1), fmaxf(e2, e3));
+                        } else {
+                            ext = neg ? INFINITY : -INFINITY;
 #pragma unroll
-                        for (int c = 0; c < 128; ++c) {
-                            const float s = __uint_as_float(sraw[c >> 5][c & 31]);
-                            const bool vis = !need_mask || (c <= lim);
-                            if (neg) ext = vis ? fminf(ext, s) : ext;
-                            else     ext = vis ? fmaxf(ext, s) : ext;
+                            for (int c = 0; c < 128; ++c) {
+                                const float s = __uint_as_float(sraw[c >> 5][c & 31]);
+                                const bool vis = !need_mask || (c <= lim);
+                                if (neg) ext = vis ? fminf(ext, s) : ext;
+                                else     ext = vis ? fmaxf(ext, s) : ext;
+                            }
                         }
-                    }
-                    const float m_tile = (fabsf(ext) == INFINITY) ? -INFINITY : ext * sl2;
-
-                    // ---- running maximum, moved lazily
-                    float alpha = 1.f;
-                    if (j == 0) {
-                        m_run = m_tile;
-                    } else if (m_tile - m_run > kRescaleThreshold) {  // also true when m_run = -inf < m_tile
-                        alpha = ex2_approx(m_run - m_tile);           // m_tile is finite here
-                        m_run = m_tile;
-                    }
-                    if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-                        // O <- alpha * O.  S_t(j) ready implies P_t V_{j-1} has finished (in-order tensor pipe).
+                        return (fabsf(ext) == INFINITY) ? -INFINITY : ext * sl2;
+                    };
+                    // p = exp2(scale*log2e*s - m) for the whole row: P -> bf16 pairs into TMEM over the
+                    // first 64 columns of S_t; returns the row sum of the fp32 probabilities.
+                    auto exp_pass = [&](float m_ref) -> float {
+                        const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+                        float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+                        const float2 sc2 = make_float2(sl2, sl2), nm2 = make_float2(neg_m, neg_m);
+#pragma unroll
+                        for (int cc = 0; cc < 4; ++cc) {
+                            uint32_t pk[16];
+#pragma unroll
+                            for (int e = 0; e < 32; e += 2) {
+                                const float2 x = __ffma2_rn(
+                                    make_float2(__uint_as_float(sraw[cc][e]), __uint_as_float(sraw[cc][e + 1])), sc2, nm2);
+                                float2 pr;
+                                if ((kFmaPipeExpMask >> ((e >> 1) & 7)) & 1) {
+                                    pr = exp2_fma_pipe(x);
+                                } else {
+                                    pr.x = ex2_approx(x.x);
+                                    pr.y = ex2_approx(x.y);
+                                }
+                                if (need_mask && generic) {
+                                    pr.x = (cc * 32 + e <= lim) ? pr.x : 0.f;
+                                    pr.y = (cc * 32 + e + 1 <= lim) ? pr.y : 0.f;
+                                }
+                                if (e & 2) acc1 = __fadd2_rn(acc1, pr);  // fp32 probabilities, before rounding to bf16
+                                else       acc0 = __fadd2_rn(acc0, pr);
+                                pk[e >> 1] = pack_bf16x2(pr.x, pr.y);
+                            }
+                            tmem_st_x16(tS + cc * 16, pk);
+                        }
+                        return (acc0.x + acc0.y) + (acc1.x + acc1.y);
+                    };
+                    // O <- alpha * O.  S_t(j) ready implies P_t V_{j-1} has finished (in-order tensor pipe).
+                    auto rescale_o = [&](float alpha) {
 #pragma unroll
                         for (int c = 0; c < D / 32; ++c) {
                             uint32_t oc[32];
@@ -576,38 +602,48 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                             for (int e = 0; e < 32; ++e) oc[e] = __float_as_uint(__uint_as_float(oc[e]) * alpha);
                             tmem_st_x32(tO + c * 32, oc);
                         }
-                    }
-                    const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
-                    if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 3);
+                    };
 
-                    // ---- p = exp2(scale*log2e*s - m); row sum in fp32; P -> bf16 pairs into TMEM
-                    float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
-                    const float2 sc2 = make_float2(sl2, sl2), nm2 = make_float2(neg_m, neg_m);
-#pragma unroll
-                    for (int cc = 0; cc < 4; ++cc) {
-                        uint32_t pk[16];
-#pragma unroll
-                        for (int e = 0; e < 32; e += 2) {
-                            const float2 x = __ffma2_rn(
-                                make_float2(__uint_as_float(sraw[cc][e]), __uint_as_float(sraw[cc][e + 1])), sc2, nm2);
-                            float2 pr;
-                            if ((kFmaPipeExpMask >> ((e >> 1) & 7)) & 1) {
-                                pr = exp2_fma_pipe(x);
-                            } else {
-                                pr.x = ex2_approx(x.x);
-                                pr.y = ex2_approx(x.y);
+                    // ---- running maximum, moved lazily: probabilities are taken relative to m_run, which
+                    // only moves when the row maximum has grown by more than the threshold
+                    float alpha = 1.f, row_sum = 0.f;
+                    // exact: take the maximum first, then exponentiate against it.  (The causal
+                    // instantiations always do: with their masking code the second copy of the
+                    // exponentiation loop costs registers and measured slower.)
+                    bool exact = CAUSAL || (j == 0);
+                    bool maximum_settled = false;
+                    if (!exact) {
+                        // Optimistic: start exponentiating against the current m_run at once and find the
+                        // tile maximum alongside; only if it exceeds m_run by more than the threshold
+                        // (rare after a row's first tiles) is O rescaled and the row redone below.
+                        const float m_tile = tile_max();
+                        row_sum = exp_pass(m_run);
+                        const bool moved = m_tile - m_run > kRescaleThreshold;  // also true for m_run = -inf < m_tile
+                        if (__any_sync(0xffffffffu, moved)) {
+                            if (moved) {
+                                alpha = ex2_approx(m_run - m_tile);  // m_tile is finite here
+                                m_run = m_tile;
                             }
-                            if (need_mask && generic) {
-                                pr.x = (cc * 32 + e <= lim) ? pr.x : 0.f;
-                                pr.y = (cc * 32 + e + 1 <= lim) ? pr.y : 0.f;
-                            }
-                            if (e & 2) acc1 = __fadd2_rn(acc1, pr);  // fp32 probabilities, before rounding to bf16
-                            else       acc0 = __fadd2_rn(acc0, pr);
-                            pk[e >> 1] = pack_bf16x2(pr.x, pr.y);
+                            rescale_o(alpha);
+                            exact = true;
+                            maximum_settled = true;
                         }
-                        tmem_st_x16(tS + cc * 16, pk);
                     }
-                    l_run = l_run * alpha + ((acc0.x + acc0.y) + (acc1.x + acc1.y));
+                    if (exact) {
+                        if (!maximum_settled) {
+                            const float m_tile = tile_max();
+                            if (j == 0) {
+                                m_run = m_tile;
+                            } else if (m_tile - m_run > kRescaleThreshold) {
+                                alpha = ex2_approx(m_run - m_tile);
+                                m_run = m_tile;
+                            }
+                            if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) rescale_o(alpha);
+                        }
+                        if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 3);
+                        row_sum = exp_pass(m_run);
+                    }
+                    l_run = l_run * alpha + row_sum;
                     if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 4);
 
                     tmem_wait_st();
