@@ -85,6 +85,32 @@ int ave_attn_fwd_host(const void *q_host, const void *k_host, const void *v_host
 size_t ave_attn_host_workspace_bytes(int B, int H, int Hkv, int Sq, int Sk, int D);
 
 /*
+ * Attention forward with the keys cut into `n_splits` ranges (split-KV): every
+ * range is processed as its own work tile with its own online softmax, and a
+ * second kernel merges the per-range results through their log-sum-exps,
+ *   LSE = ln sum_s exp(LSE_s),   O = sum_s exp(LSE_s - LSE) * O_s,
+ * which is the same re-association of the softmax sum that the tiling of paper
+ * Section 2 relies on, applied across CTAs.  Same tensors, layouts, limits and
+ * result as ave_attn_fwd (up to rounding order); meant for few query rows
+ * against many keys (decode, chunked prefill), where one work tile per
+ * (batch, head, 256 query rows) would leave most SMs idle.
+ * n_splits: 1 .. AVE_SPLITKV_MAX_SPLITS; each range is ceil(Sk / n_splits)
+ * keys rounded up to a multiple of 128 (trailing ranges may be empty).
+ * workspace: DEVICE scratch of at least ave_attn_splitkv_workspace_bytes(...)
+ * bytes, 256-byte aligned, owned by the caller; it holds the fp32 partial
+ * outputs and log-sum-exps, is fully rewritten by each call, and may be
+ * reused by later calls on the same stream.  Two kernels are enqueued.
+ */
+#define AVE_SPLITKV_MAX_SPLITS 64
+int ave_attn_fwd_splitkv(const void *q, const void *k, const void *v, void *o, float *lse,
+                         int B, int H, int Hkv, int Sq, int Sk, int D,
+                         int causal, float scale, int n_splits,
+                         void *workspace, size_t workspace_bytes, void *stream);
+
+/* Bytes of device workspace ave_attn_fwd_splitkv needs; 0 if an argument is invalid. */
+size_t ave_attn_splitkv_workspace_bytes(int B, int H, int Sq, int D, int n_splits);
+
+/*
  * Synchronises the current device, then reads and clears the device-side
  * status word that kernels set when one of their bounded waits (on an
  * mbarrier) runs out.  Returns AVE_OK, AVE_ERR_DEVICE_TIMEOUT (with the raw

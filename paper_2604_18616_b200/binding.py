@@ -51,6 +51,10 @@ def lib() -> ctypes.CDLL:
         L.ave_attn_fwd_host.restype = ci
         L.ave_attn_host_workspace_bytes.argtypes = [ci] * 6
         L.ave_attn_host_workspace_bytes.restype = ctypes.c_size_t
+        L.ave_attn_fwd_splitkv.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, cf, ci, vp, ctypes.c_size_t, vp]
+        L.ave_attn_fwd_splitkv.restype = ci
+        L.ave_attn_splitkv_workspace_bytes.argtypes = [ci] * 5
+        L.ave_attn_splitkv_workspace_bytes.restype = ctypes.c_size_t
         L.ave_attn_device_status.argtypes = [ctypes.POINTER(ctypes.c_uint)]
         L.ave_attn_device_status.restype = ci
         L.ave_attn_launch_count.argtypes = []
@@ -154,4 +158,34 @@ def ave_attn_fwd_host(q, k, v, o, lse, workspace, causal=False, scale=None, stre
             _stream_ptr(stream))
     if st != AVE_OK:
         raise AveAttnError(st, "ave_attn_fwd_host")
+    return o, lse
+
+
+def splitkv_workspace_bytes(B, H, Sq, D, n_splits) -> int:
+    return int(lib().ave_attn_splitkv_workspace_bytes(B, H, Sq, D, n_splits))
+
+
+def ave_attn_fwd_splitkv(q, k, v, n_splits, workspace=None, o=None, lse=None, causal=False, scale=None, stream=None):
+    """Split-KV variant of ``ave_attn_fwd``: same tensors and result; ``workspace``
+    is a CUDA uint8 tensor of at least ``splitkv_workspace_bytes`` bytes
+    (allocated here when not given)."""
+    B, H, Sq, D = q.shape
+    _, Hkv, Sk, _ = k.shape
+    if o is None:
+        o = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((B, H, Sq), dtype=torch.float32, device=q.device)
+    if scale is None:
+        scale = D ** -0.5
+    if workspace is None:
+        workspace = torch.empty(max(256, splitkv_workspace_bytes(B, H, Sq, D, n_splits)), dtype=torch.uint8,
+                                device=q.device)
+    with torch.cuda.device(q.device):
+        st = lib().ave_attn_fwd_splitkv(
+            ctypes.c_void_p(q.data_ptr()), ctypes.c_void_p(k.data_ptr()), ctypes.c_void_p(v.data_ptr()),
+            ctypes.c_void_p(o.data_ptr()), ctypes.c_void_p(lse.data_ptr()),
+            B, H, Hkv, Sq, Sk, D, int(bool(causal)), float(scale), int(n_splits),
+            ctypes.c_void_p(workspace.data_ptr()), ctypes.c_size_t(workspace.numel()), _stream_ptr(stream))
+    if st != AVE_OK:
+        raise AveAttnError(st, "ave_attn_fwd_splitkv")
     return o, lse

@@ -38,6 +38,13 @@ struct FwdParams {
     int total_blocks; // n_qblk * BH = grid size
     int heads_per_group;  // (b, h) pairs whose work tiles are launched together (their K/V share L2)
     float scale_log2; // scale * log2(e)
+    int causal_off;   // key j is visible to query i iff j <= i + causal_off (Sk - Sq of the whole problem)
+    // Split-KV launches only: the keys are cut into n_splits ranges of keys_per_split (a multiple of
+    // BN); a work tile handles one range and writes a normalised fp32 partial result.
+    int n_splits;
+    int keys_per_split;
+    float *o_partial;    // fp32 [n_splits, B*H, Sq, D]
+    float *lse_partial;  // fp32 [n_splits, B*H, Sq]
 };
 
 // tcgen05 instruction descriptor, kind::f16: fp32 accumulator, bf16 A and B,

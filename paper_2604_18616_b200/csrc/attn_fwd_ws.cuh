@@ -79,16 +79,32 @@ __device__ __forceinline__ void setmaxnreg_dec() {
 }
 
 // One work tile, decoded from its position in the launch order.
-struct WorkTile {
+struct WorkTileBase {
     int bh;      // b * H + h
     int bg;      // b * Hkv + h / (H / Hkv): key/value head (Fig. 1: idx_h / gqa)
     int q0;      // first query row
     int n0, n1;  // key tiles the two sub-tiles visit (n1 >= n0)
 };
+template <bool SPLIT>
+struct WorkTileT : WorkTileBase {};
+template <>
+struct WorkTileT<true> : WorkTileBase {
+    int k_begin, k_end;  // keys [k_begin, k_end) belong to this tile (split-KV only; else the whole range)
+    int split;           // index of the key range
+};
 
-// Number of key tiles a 128-row sub-tile starting at row i0 must visit.
+// Number of key tiles a 128-row sub-tile starting at row i0 must visit inside [k_begin, k_end).
 template <bool CAUSAL>
-__device__ __forceinline__ int kv_tiles_for(int i0, int Sq, int Sk) {
+__device__ __forceinline__ int kv_tiles_for(int i0, int causal_off, int k_begin, int k_end) {
+    int hi = k_end;
+    if (CAUSAL) hi = min(hi, i0 + BM + causal_off);  // one past the last key the sub-tile's last row may see
+    return hi > k_begin ? (hi - k_begin + BN - 1) / BN : 0;
+}
+
+// The same count when the tile covers all keys [0, Sk): key j is visible to row i iff
+// j <= i + (Sk - Sq).
+template <bool CAUSAL>
+__device__ __forceinline__ int kv_tiles_whole(int i0, int Sq, int Sk) {
     int n = (Sk + BN - 1) / BN;
     if (CAUSAL) {
         const int last_vis = i0 + BM - 1 + (Sk - Sq);  // last key the last row of the sub-tile may see
@@ -99,26 +115,46 @@ __device__ __forceinline__ int kv_tiles_for(int i0, int Sq, int Sk) {
 
 // Launch order: (batch, head) pairs in groups of p.heads_per_group (whose K/V
 // fit in L2 together); inside a group all heads' blocks of one query position,
-// longest (causal: last) position first.
-template <bool CAUSAL>
-__device__ __forceinline__ WorkTile decode_tile(int id, const FwdParams &p) {
+// longest (causal: last) position first.  Split-KV: the key ranges of one
+// (b, h, block) are adjacent in the order.
+template <bool CAUSAL, bool SPLIT>
+__device__ __forceinline__ WorkTileT<SPLIT> decode_tile(int id, const FwdParams &p) {
+    WorkTileT<SPLIT> w;
+    int k_begin = 0, k_end = p.Sk;
+    if constexpr (SPLIT) {
+        w.split = id % p.n_splits;
+        id /= p.n_splits;
+        w.k_begin = k_begin = min(p.Sk, w.split * p.keys_per_split);
+        w.k_end = k_end = min(p.Sk, w.k_begin + p.keys_per_split);
+    }
     const int per_group = p.heads_per_group * p.n_qblk;
     const int grp = id / per_group;
     const int rem = id - grp * per_group;
     const int bh0 = grp * p.heads_per_group;
     const int hg = min(p.heads_per_group, p.BH - bh0);
     const int rank = rem / hg;
-    WorkTile w;
     w.bh = bh0 + (rem - rank * hg);
     const int qb = CAUSAL ? (p.n_qblk - 1 - rank) : rank;
     const int b = w.bh / p.H;
     const int h = w.bh - b * p.H;
     w.bg = b * p.Hkv + h / (p.H / p.Hkv);
     w.q0 = qb * 2 * BM;
-    w.n0 = kv_tiles_for<CAUSAL>(w.q0, p.Sq, p.Sk);
-    w.n1 = kv_tiles_for<CAUSAL>(w.q0 + BM, p.Sq, p.Sk);
+    if constexpr (SPLIT) {
+        w.n0 = kv_tiles_for<CAUSAL>(w.q0, p.causal_off, k_begin, k_end);
+        w.n1 = kv_tiles_for<CAUSAL>(w.q0 + BM, p.causal_off, k_begin, k_end);
+    } else {
+        w.n0 = kv_tiles_whole<CAUSAL>(w.q0, p.Sq, p.Sk);
+        w.n1 = kv_tiles_whole<CAUSAL>(w.q0 + BM, p.Sq, p.Sk);
+    }
     return w;
 }
+
+__device__ __forceinline__ int key_begin(const WorkTileT<false> &) { return 0; }
+__device__ __forceinline__ int key_begin(const WorkTileT<true> &w) { return w.k_begin; }
+__device__ __forceinline__ int key_end(const WorkTileT<false> &, const FwdParams &p) { return p.Sk; }
+__device__ __forceinline__ int key_end(const WorkTileT<true> &w, const FwdParams &) { return w.k_end; }
+__device__ __forceinline__ int split_of(const WorkTileT<false> &) { return 0; }
+__device__ __forceinline__ int split_of(const WorkTileT<true> &w) { return w.split; }
 
 // ---- cluster launch control: take over the tile of a CTA that has not started
 __device__ __forceinline__ void clc_try_cancel(uint32_t response_smem, uint32_t bar) {
@@ -144,7 +180,7 @@ __device__ __forceinline__ int clc_decode(const volatile unsigned long long *res
     return ok ? int(x) : -1;
 }
 
-template <int D, bool CAUSAL>
+template <int D, bool CAUSAL, bool SPLIT>
 __global__ void __launch_bounds__(384, 1)
 attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
@@ -256,7 +292,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             bool ok = true;
             int id = blockIdx.x;
             for (int n = 0; id >= 0 && ok; ++n) {
-                const WorkTile w = decode_tile<CAUSAL>(id, p);
+                const WorkTileT<SPLIT> w = decode_tile<CAUSAL, SPLIT>(id, p);
                 // Q_t of this tile goes in as soon as the previous tile's last Q_t K^T has retired.
                 // Q_1 is released later than Q_0 (causal sub-tile 1 runs one step longer), and the
                 // first K/V tiles must not queue behind it, so a Q load that cannot go yet stays
@@ -317,7 +353,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         mbar_arrive_expect_tx(bar, Cfg::kTileBytes);
                         for (int x = 0; x < Cfg::kBoxes; ++x)
                             tma_load_3d(sRing + slot * Cfg::kTileBytes + x * Cfg::kBoxBytes, tm, bar, x * 64,
-                                        (it >> 1) * BN, w.bg);
+                                        key_begin(w) + (it >> 1) * BN, w.bg);
                     }
                 }
                 if (ok) try_load_q(0, true);
@@ -375,7 +411,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             // First step of sub-tile t in tile number `tn` (tile `wt`, whose K_0 sits at ring position
             // `ring0`): S_t = Q_t K_0^T.  Issued as soon as sub-tile t has finished the tile before, so
             // the next tile's first scores are computed while the other sub-tile is still at work.
-            auto start_subtile = [&](int t, const WorkTile &wt, int tn, int ring0) {
+            auto start_subtile = [&](int t, const WorkTileT<SPLIT> &wt, int tn, int ring0) {
                 const int n_t = t ? wt.n1 : wt.n0;
                 ok = wait_bar(&bar_q_full[t], tn & 1, STATUS_TIMEOUT_LOAD);
                 if (ok && n_t > 0) ok = wait_full(ring0);
@@ -391,7 +427,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             };
 
             int id = blockIdx.x;
-            WorkTile w = decode_tile<CAUSAL>(id, p);
+            WorkTileT<SPLIT> w = decode_tile<CAUSAL, SPLIT>(id, p);
             start_subtile(0, w, 0, 0);
             if (ok) start_subtile(1, w, 0, 0);
             for (int n = 0; id >= 0 && ok; ++n) {
@@ -400,8 +436,8 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 // the tile after this one (its first steps are issued from inside this tile's loop)
                 const int id_next = next_tile(n, ok);
                 if (!ok) break;
-                WorkTile w_next = w;
-                if (id_next >= 0) w_next = decode_tile<CAUSAL>(id_next, p);
+                WorkTileT<SPLIT> w_next = w;
+                if (id_next >= 0) w_next = decode_tile<CAUSAL, SPLIT>(id_next, p);
                 const int ring_next = ring + 2 * n1;
                 if (id_next >= 0 && n1 == 0) {  // nothing to do in this tile at all
                     start_subtile(0, w_next, n + 1, ring_next);
@@ -472,7 +508,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const int t = (warp - 4) >> 2;                // sub-tile
         const int wq = warp & 3;                      // TMEM lane quadrant of this warp
         const int r = wq * 32 + lane;                 // row within the sub-tile = TMEM lane
-        const int off = p.Sk - p.Sq;
+        const int off = SPLIT ? p.causal_off : p.Sk - p.Sq;
         const uint32_t lane_sel = uint32_t(wq * 32) << 16;
         const uint32_t tS = tmem + (t ? Cfg::kColS1 : Cfg::kColS0) + lane_sel;
         const uint32_t tO = tmem + (t ? Cfg::kColO1 : Cfg::kColO0) + lane_sel;
@@ -487,7 +523,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 
         int id = blockIdx.x;
         for (int n = 0; id >= 0 && ok; ++n) {
-            const WorkTile w = decode_tile<CAUSAL>(id, p);
+            const WorkTileT<SPLIT> w = decode_tile<CAUSAL, SPLIT>(id, p);
             const int bh = w.bh;
             const int i0 = w.q0 + t * BM;
             const int i = i0 + r;                     // query row
@@ -496,10 +532,16 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             if (n_t == 0) {
                 // no key visible to any row of this sub-tile: O = 0, LSE = -inf
                 if (i < p.Sq) {
-                    __nv_bfloat16 *o_row = reinterpret_cast<__nv_bfloat16 *>(p.o) + (size_t(bh) * p.Sq + i) * D;
                     const uint4 z = make_uint4(0, 0, 0, 0);
-                    for (int c = 0; c < D / 8; ++c) reinterpret_cast<uint4 *>(o_row)[c] = z;
-                    p.lse[size_t(bh) * p.Sq + i] = -INFINITY;
+                    if (SPLIT) {
+                        const size_t row = (size_t(split_of(w)) * p.BH + bh) * p.Sq + i;
+                        for (int c = 0; c < D / 4; ++c) reinterpret_cast<uint4 *>(p.o_partial + row * D)[c] = z;
+                        p.lse_partial[row] = -INFINITY;
+                    } else {
+                        __nv_bfloat16 *o_row = reinterpret_cast<__nv_bfloat16 *>(p.o) + (size_t(bh) * p.Sq + i) * D;
+                        for (int c = 0; c < D / 8; ++c) reinterpret_cast<uint4 *>(o_row)[c] = z;
+                        p.lse[size_t(bh) * p.Sq + i] = -INFINITY;
+                    }
                 }
                 // O_t was not used: hand it back at once so its barrier completes once per tile
                 __syncwarp();
@@ -519,10 +561,11 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     tmem_wait_ld();
                     if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 2);
 
-                    const int j0 = j * BN;
-                    int lim = p.Sk - 1 - j0;  // columns c <= lim of this tile are visible to row i
+                    const int k_end = key_end(w, p);
+                    const int j0 = key_begin(w) + j * BN;  // first key of this step
+                    int lim = k_end - 1 - j0;           // columns c <= lim of this tile are visible to row i
                     if (CAUSAL) lim = min(lim, i + off - j0);
-                    const bool need_mask = (j0 + BN > p.Sk) || (CAUSAL && (j0 + BN - 1 > i0 + off));
+                    const bool need_mask = (j0 + BN > k_end) || (CAUSAL && (j0 + BN - 1 > i0 + off));
 
                     // ---- row extreme of the raw scores (maximum of scale*s is at max s, or min s if scale < 0)
                     // With a positive scale a masked score is simply replaced by -inf: it then drops out
@@ -659,9 +702,29 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     ++n_out;
                     tc_fence_after();
                     const float inv_l = (l_run > 0.f) ? 1.f / l_run : 0.f;
-                    if (i < p.Sq)
-                        p.lse[size_t(bh) * p.Sq + i] =
-                            (l_run > 0.f) ? (m_run + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+                    const float lse_row = (l_run > 0.f) ? (m_run + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+                    if (SPLIT) {
+                        // partial result of this key range: normalised O in fp32 and its LSE, straight to global
+                        const size_t row = (size_t(split_of(w)) * p.BH + bh) * p.Sq + i;
+                        if (i < p.Sq) p.lse_partial[row] = lse_row;
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t oc[32];
+                            tmem_ld_x32(tO + c * 32, oc);
+                            tmem_wait_ld();
+                            if (i < p.Sq) {
+#pragma unroll
+                                for (int e = 0; e < 32; e += 4)
+                                    reinterpret_cast<float4 *>(p.o_partial + row * D + c * 32)[e >> 2] =
+                                        make_float4(__uint_as_float(oc[e]) * inv_l, __uint_as_float(oc[e + 1]) * inv_l,
+                                                    __uint_as_float(oc[e + 2]) * inv_l, __uint_as_float(oc[e + 3]) * inv_l);
+                            }
+                        }
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&bar_o_free[t]));
+                    } else {
+                    if (i < p.Sq) p.lse[size_t(bh) * p.Sq + i] = lse_row;
 #pragma unroll
                     for (int x = 0; x < Cfg::kBoxes; ++x) {  // 64 columns of O at a time through the staging rows
                         uint32_t oc[2][32];
@@ -697,6 +760,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                             tma_store_commit();
                             store_pending = true;
                         }
+                    }
                     }
                 }
             }

@@ -105,11 +105,11 @@ int check_device() {
     return AVE_OK;
 }
 
-template <int D, bool CAUSAL>
+template <int D, bool CAUSAL, bool SPLIT>
 int launch_ws(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const CUtensorMap &to,
               const ave::FwdParams &p, cudaStream_t stream) {
     using Cfg = ave::WsCfg<D>;
-    auto kern = ave::attn_fwd_ws_kernel<D, CAUSAL>;
+    auto kern = ave::attn_fwd_ws_kernel<D, CAUSAL, SPLIT>;
     static std::atomic<bool> configured{false};  // per instantiation
     if (!configured.load(std::memory_order_acquire)) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
@@ -120,6 +120,123 @@ int launch_ws(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &t
         configured.store(true, std::memory_order_release);
     }
     kern<<<dim3(p.total_blocks), dim3(Cfg::kThreads), Cfg::kSmemBytes, stream>>>(tq, tk, tv, to, p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        t_last_cuda_error = int(e);
+        return AVE_ERR_CUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return AVE_OK;
+}
+
+
+// Encode the tensor maps, fill the kernel parameters and launch.  n_splits == 1 with no partial
+// buffers is the ordinary forward; otherwise every work tile covers one range of keys_per_split keys
+// and writes fp32 partials.
+int launch_attention(const void *q, const void *k, const void *v, void *o, float *lse, int B, int H, int Hkv, int Sq,
+                     int Sk, int D, int causal, float scale, int n_splits, int keys_per_split, float *o_partial,
+                     float *lse_partial, cudaStream_t s) {
+    CUtensorMap tq, tk, tv, to;
+    if (!encode_map(&tq, q, D, Sq, (long long)B * H, ave::BM)) return AVE_ERR_CUDA;
+    if (!encode_map(&to, o, D, Sq, (long long)B * H, ave::WsCfg<128>::kOutBoxRows)) return AVE_ERR_CUDA;
+    if (!encode_map(&tk, k, D, Sk, (long long)B * Hkv, ave::BN)) return AVE_ERR_CUDA;
+    if (!encode_map(&tv, v, D, Sk, (long long)B * Hkv, ave::BN)) return AVE_ERR_CUDA;
+
+    const bool split = o_partial != nullptr;
+    ave::FwdParams p;
+    p.o = o;
+    p.lse = lse;
+    p.H = H;
+    p.Hkv = Hkv;
+    p.Sq = Sq;
+    p.Sk = Sk;
+    p.BH = B * H;
+    p.n_qblk = (Sq + 2 * ave::BM - 1) / (2 * ave::BM);
+    p.causal_off = Sk - Sq;
+    p.n_splits = split ? n_splits : 1;
+    p.keys_per_split = split ? keys_per_split : Sk;
+    p.o_partial = o_partial;
+    p.lse_partial = lse_partial;
+    const long long total = (long long)p.n_qblk * p.BH * p.n_splits;
+    if (total >= (1ll << 31)) return AVE_ERR_BAD_SHAPE;
+    p.total_blocks = int(total);
+    {
+        // Launch (b, h) pairs in groups whose K and V together stay within a slice of L2,
+        // whole key/value heads at a time.
+        const long long kv_bytes_per_kv_head = 2ll * Sk * D * 2;
+        const int G = H / Hkv;
+        const long long budget = 64ll << 20;
+        long long kv_heads = budget / kv_bytes_per_kv_head;
+        if (kv_heads < 1) kv_heads = 1;
+        long long hpg = kv_heads * G;
+        if (hpg > p.BH) hpg = p.BH;
+        p.heads_per_group = int(hpg);
+    }
+    p.scale_log2 = scale * 1.4426950408889634f;
+
+    if (split) {
+        if (D == 128)
+            return causal ? launch_ws<128, true, true>(tq, tk, tv, to, p, s) : launch_ws<128, false, true>(tq, tk, tv, to, p, s);
+        return causal ? launch_ws<64, true, true>(tq, tk, tv, to, p, s) : launch_ws<64, false, true>(tq, tk, tv, to, p, s);
+    }
+    if (D == 128)
+        return causal ? launch_ws<128, true, false>(tq, tk, tv, to, p, s) : launch_ws<128, false, false>(tq, tk, tv, to, p, s);
+    return causal ? launch_ws<64, true, false>(tq, tk, tv, to, p, s) : launch_ws<64, false, false>(tq, tk, tv, to, p, s);
+}
+
+// Combine the partial results of the key ranges of every query row:
+//   LSE = ln sum_s exp(LSE_s),  O = sum_s exp(LSE_s - LSE) * O_s.
+// One thread per (row, 8 output columns).
+__global__ void splitkv_merge_kernel(const float *__restrict__ o_partial, const float *__restrict__ lse_partial,
+                                     __nv_bfloat16 *__restrict__ o, float *__restrict__ lse, long long rows, int D,
+                                     int n_splits) {
+    const int chunks = D / 8;
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= rows * chunks) return;
+    const long long row = idx / chunks;
+    const int ch = int(idx - row * chunks);
+    float m = -INFINITY;
+    for (int s = 0; s < n_splits; ++s) m = fmaxf(m, lse_partial[s * rows + row]);
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    float denom = 0.f;
+    if (m != -INFINITY) {
+        for (int s = 0; s < n_splits; ++s) {
+            const float w = __expf(lse_partial[s * rows + row] - m);
+            denom += w;
+            const float4 *src = reinterpret_cast<const float4 *>(o_partial + (s * rows + row) * D + ch * 8);
+            const float4 a = src[0], b = src[1];
+            acc[0] += w * a.x; acc[1] += w * a.y; acc[2] += w * a.z; acc[3] += w * a.w;
+            acc[4] += w * b.x; acc[5] += w * b.y; acc[6] += w * b.z; acc[7] += w * b.w;
+        }
+    }
+    const float inv = denom > 0.f ? 1.f / denom : 0.f;
+    uint4 out;
+    out.x = ave::pack_bf16x2(acc[0] * inv, acc[1] * inv);
+    out.y = ave::pack_bf16x2(acc[2] * inv, acc[3] * inv);
+    out.z = ave::pack_bf16x2(acc[4] * inv, acc[5] * inv);
+    out.w = ave::pack_bf16x2(acc[6] * inv, acc[7] * inv);
+    reinterpret_cast<uint4 *>(o + row * D)[ch] = out;
+    if (ch == 0) lse[row] = (denom > 0.f) ? m + logf(denom) : -INFINITY;
+}
+
+// Keys per range: an equal share of Sk rounded up to whole key tiles.
+int splitkv_keys_per_split(int Sk, int n_splits) {
+    const long long share = ((long long)Sk + n_splits - 1) / n_splits;
+    return int((share + ave::BN - 1) / ave::BN * ave::BN);
+}
+
+int run_splitkv(const void *q, const void *k, const void *v, void *o, float *lse, int B, int H, int Hkv, int Sq,
+                int Sk, int D, int causal, float scale, int n_splits, float *o_partial, float *lse_partial,
+                cudaStream_t s) {
+    const int kps = splitkv_keys_per_split(Sk, n_splits);
+    int st = launch_attention(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, causal, scale, n_splits, kps, o_partial,
+                              lse_partial, s);
+    if (st != AVE_OK) return st;
+    const long long rows = (long long)B * H * Sq;
+    const long long work = rows * (D / 8);
+    const int threads = 256;
+    splitkv_merge_kernel<<<unsigned((work + threads - 1) / threads), threads, 0, s>>>(
+        o_partial, lse_partial, static_cast<__nv_bfloat16 *>(o), lse, rows, D, n_splits);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
         t_last_cuda_error = int(e);
@@ -141,41 +258,8 @@ int ave_attn_fwd(const void *q, const void *k, const void *v, void *o, float *ls
     if (st != AVE_OK) return st;
     st = check_device();
     if (st != AVE_OK) return st;
-
-    CUtensorMap tq, tk, tv, to;
-    if (!encode_map(&tq, q, D, Sq, (long long)B * H, ave::BM)) return AVE_ERR_CUDA;
-    if (!encode_map(&to, o, D, Sq, (long long)B * H, ave::WsCfg<128>::kOutBoxRows)) return AVE_ERR_CUDA;
-    if (!encode_map(&tk, k, D, Sk, (long long)B * Hkv, ave::BN)) return AVE_ERR_CUDA;
-    if (!encode_map(&tv, v, D, Sk, (long long)B * Hkv, ave::BN)) return AVE_ERR_CUDA;
-
-    ave::FwdParams p;
-    p.o = o;
-    p.lse = lse;
-    p.H = H;
-    p.Hkv = Hkv;
-    p.Sq = Sq;
-    p.Sk = Sk;
-    p.BH = B * H;
-    p.n_qblk = (Sq + 2 * ave::BM - 1) / (2 * ave::BM);
-    p.total_blocks = p.n_qblk * p.BH;
-    {
-        // Launch (b, h) pairs in groups whose K and V together stay within a slice of L2,
-        // whole key/value heads at a time.
-        const long long kv_bytes_per_kv_head = 2ll * Sk * D * 2;
-        const int G = H / Hkv;
-        const long long budget = 64ll << 20;
-        long long kv_heads = budget / kv_bytes_per_kv_head;
-        if (kv_heads < 1) kv_heads = 1;
-        long long hpg = kv_heads * G;
-        if (hpg > p.BH) hpg = p.BH;
-        p.heads_per_group = int(hpg);
-    }
-    p.scale_log2 = scale * 1.4426950408889634f;
-
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (D == 128)
-        return causal ? launch_ws<128, true>(tq, tk, tv, to, p, s) : launch_ws<128, false>(tq, tk, tv, to, p, s);
-    return causal ? launch_ws<64, true>(tq, tk, tv, to, p, s) : launch_ws<64, false>(tq, tk, tv, to, p, s);
+    return launch_attention(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, causal, scale, 1, 0, nullptr, nullptr,
+                            static_cast<cudaStream_t>(stream));
 }
 
 size_t ave_attn_host_workspace_bytes(int B, int H, int Hkv, int Sq, int Sk, int D) {
@@ -224,6 +308,33 @@ int ave_attn_fwd_host(const void *q_host, const void *k_host, const void *v_host
         return AVE_ERR_CUDA;
     }
     return AVE_OK;
+}
+
+size_t ave_attn_splitkv_workspace_bytes(int B, int H, int Sq, int D, int n_splits) {
+    if (B <= 0 || H <= 0 || Sq <= 0 || (D != 64 && D != 128) || n_splits < 1 || n_splits > AVE_SPLITKV_MAX_SPLITS)
+        return 0;
+    const size_t rows = size_t(B) * H * Sq;
+    return size_t(n_splits) * rows * (size_t(D) + 1) * sizeof(float);
+}
+
+int ave_attn_fwd_splitkv(const void *q, const void *k, const void *v, void *o, float *lse, int B, int H, int Hkv,
+                         int Sq, int Sk, int D, int causal, float scale, int n_splits, void *workspace,
+                         size_t workspace_bytes, void *stream) {
+    int st = validate(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, scale);
+    if (st >= 0) return st;
+    if (n_splits < 1 || n_splits > AVE_SPLITKV_MAX_SPLITS) return AVE_ERR_BAD_SHAPE;
+    st = validate_ptrs_and_scale(q, k, v, o, lse, scale);
+    if (st != AVE_OK) return st;
+    const size_t need = ave_attn_splitkv_workspace_bytes(B, H, Sq, D, n_splits);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < need)
+        return AVE_ERR_WORKSPACE;
+    st = check_device();
+    if (st != AVE_OK) return st;
+    const size_t rows = size_t(B) * H * Sq;
+    float *o_partial = static_cast<float *>(workspace);
+    float *lse_partial = o_partial + size_t(n_splits) * rows * D;
+    return run_splitkv(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, causal, scale, n_splits, o_partial, lse_partial,
+                       static_cast<cudaStream_t>(stream));
 }
 
 int ave_attn_device_status(unsigned int *raw_word) {
