@@ -42,7 +42,8 @@ typedef enum {
     AVE_ERR_UNSUPPORTED_DEVICE = 6, /* the current device is not compute capability 10.x */
     AVE_ERR_CUDA = 7,               /* a CUDA call failed; see ave_attn_last_cuda_error() */
     AVE_ERR_DEVICE_TIMEOUT = 8,     /* a bounded wait inside a kernel gave up (ave_attn_device_status) */
-    AVE_ERR_WORKSPACE = 9           /* workspace NULL, misaligned or too small */
+    AVE_ERR_WORKSPACE = 9,          /* workspace NULL, misaligned or too small */
+    AVE_ERR_STATIC_SCRATCH = 10     /* the problem needs more scratch than the library's built-in array holds */
 } ave_status_t;
 
 /*
@@ -109,6 +110,41 @@ int ave_attn_fwd_splitkv(const void *q, const void *k, const void *v, void *o, f
 
 /* Bytes of device workspace ave_attn_fwd_splitkv needs; 0 if an argument is invalid. */
 size_t ave_attn_splitkv_workspace_bytes(int B, int H, int Sq, int D, int n_splits);
+
+/*
+ * Split-KV attention for callers that must not allocate device memory.
+ * (The paper has no counterpart to this entry point; it exists for deployment
+ * reasons only.)
+ *
+ * Some hosts of this library cannot hand it a workspace: an inference server
+ * that reserved all device memory for its KV cache at start-up, a real-time
+ * loop in which a cudaMalloc (which may synchronise the whole device) is not
+ * acceptable, or a plug-in whose host application owns the allocator.  For
+ * them this variant of ave_attn_fwd_splitkv keeps its scratch (the fp32
+ * partial outputs and log-sum-exps of the key ranges) in an array that is
+ * part of the library's device image: AVE_SPLITKV_STATIC_SCRATCH_BYTES bytes
+ * on every GPU that loads the library, held until the process exits.  The
+ * call itself performs no cudaMalloc/cudaFree and calls no allocating
+ * routine; inputs and outputs are still the caller's.
+ *
+ * Same arguments, layouts and result as ave_attn_fwd_splitkv without the
+ * workspace.  A problem whose scratch need,
+ * ave_attn_splitkv_workspace_bytes(B, H, Sq, D, n_splits), exceeds
+ * AVE_SPLITKV_STATIC_SCRATCH_BYTES is rejected with AVE_ERR_STATIC_SCRATCH
+ * and nothing is launched (use fewer ranges, or the workspace variant).
+ *
+ * The first call on each device looks up the array's device address (with
+ * that device current) and remembers it; make that first call outside any
+ * stream capture.  All calls on a device share the one array: it keeps the
+ * previous call's contents, which is harmless because every call rewrites all
+ * the partials it later reads (nothing has to start at zero), but two calls
+ * that overlap on the GPU (different streams, no dependency) race on it and
+ * give wrong results.  Serialise such calls.
+ */
+#define AVE_SPLITKV_STATIC_SCRATCH_BYTES (8u << 20)
+int ave_attn_fwd_splitkv_static(const void *q, const void *k, const void *v, void *o, float *lse,
+                                int B, int H, int Hkv, int Sq, int Sk, int D,
+                                int causal, float scale, int n_splits, void *stream);
 
 /*
  * Synchronises the current device, then reads and clears the device-side

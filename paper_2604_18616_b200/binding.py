@@ -24,6 +24,8 @@ AVE_ERR_UNSUPPORTED_DEVICE = 6
 AVE_ERR_CUDA = 7
 AVE_ERR_DEVICE_TIMEOUT = 8
 AVE_ERR_WORKSPACE = 9
+AVE_ERR_STATIC_SCRATCH = 10
+SPLITKV_STATIC_SCRATCH_BYTES = 8 << 20
 
 _lib = None
 
@@ -53,6 +55,8 @@ def lib() -> ctypes.CDLL:
         L.ave_attn_host_workspace_bytes.restype = ctypes.c_size_t
         L.ave_attn_fwd_splitkv.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, cf, ci, vp, ctypes.c_size_t, vp]
         L.ave_attn_fwd_splitkv.restype = ci
+        L.ave_attn_fwd_splitkv_static.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, cf, ci, vp]
+        L.ave_attn_fwd_splitkv_static.restype = ci
         L.ave_attn_splitkv_workspace_bytes.argtypes = [ci] * 5
         L.ave_attn_splitkv_workspace_bytes.restype = ctypes.c_size_t
         L.ave_attn_device_status.argtypes = [ctypes.POINTER(ctypes.c_uint)]
@@ -188,4 +192,25 @@ def ave_attn_fwd_splitkv(q, k, v, n_splits, workspace=None, o=None, lse=None, ca
             ctypes.c_void_p(workspace.data_ptr()), ctypes.c_size_t(workspace.numel()), _stream_ptr(stream))
     if st != AVE_OK:
         raise AveAttnError(st, "ave_attn_fwd_splitkv")
+    return o, lse
+
+
+def ave_attn_fwd_splitkv_static(q, k, v, n_splits, o, lse, causal=False, scale=None, stream=None):
+    """Split-KV attention for callers that must not allocate device memory
+    (servers that reserved all of it up front, latency-critical loops, plug-ins
+    whose host owns the allocator): the scratch is an array built into the
+    library, ``SPLITKV_STATIC_SCRATCH_BYTES`` per GPU.  ``o`` and ``lse`` must be
+    passed in, so this wrapper allocates nothing either.  Calls sharing a
+    device must not overlap on the GPU."""
+    B, H, Sq, D = q.shape
+    _, Hkv, Sk, _ = k.shape
+    if scale is None:
+        scale = D ** -0.5
+    with torch.cuda.device(q.device):
+        st = lib().ave_attn_fwd_splitkv_static(
+            ctypes.c_void_p(q.data_ptr()), ctypes.c_void_p(k.data_ptr()), ctypes.c_void_p(v.data_ptr()),
+            ctypes.c_void_p(o.data_ptr()), ctypes.c_void_p(lse.data_ptr()),
+            B, H, Hkv, Sq, Sk, D, int(bool(causal)), float(scale), int(n_splits), _stream_ptr(stream))
+    if st != AVE_OK:
+        raise AveAttnError(st, "ave_attn_fwd_splitkv_static")
     return o, lse

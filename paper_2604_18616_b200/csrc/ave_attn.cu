@@ -14,6 +14,11 @@
 
 #include "attn_fwd_ws.cuh"
 
+// Scratch of ave_attn_fwd_splitkv_static: part of the device image, so every GPU that loads the
+// library holds it until exit.  In host code this name is only a handle for
+// cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_splitkv_static_scratch[AVE_SPLITKV_STATIC_SCRATCH_BYTES];
+
 namespace {
 
 thread_local int t_last_cuda_error = 0;
@@ -337,6 +342,44 @@ int ave_attn_fwd_splitkv(const void *q, const void *k, const void *v, void *o, f
                        static_cast<cudaStream_t>(stream));
 }
 
+int ave_attn_fwd_splitkv_static(const void *q, const void *k, const void *v, void *o, float *lse, int B, int H,
+                                int Hkv, int Sq, int Sk, int D, int causal, float scale, int n_splits,
+                                void *stream) {
+    int st = validate(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, scale);
+    if (st >= 0) return st;
+    if (n_splits < 1 || n_splits > AVE_SPLITKV_MAX_SPLITS) return AVE_ERR_BAD_SHAPE;
+    st = validate_ptrs_and_scale(q, k, v, o, lse, scale);
+    if (st != AVE_OK) return st;
+    const size_t need = ave_attn_splitkv_workspace_bytes(B, H, Sq, D, n_splits);
+    if (need == 0 || need > size_t(AVE_SPLITKV_STATIC_SCRATCH_BYTES)) return AVE_ERR_STATIC_SCRATCH;
+    st = check_device();
+    if (st != AVE_OK) return st;
+
+    // Device address of the built-in array, looked up once per device with that device current.
+    constexpr int kMaxDevices = 64;
+    static std::atomic<void *> scratch_of_device[kMaxDevices];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        t_last_cuda_error = int(e != cudaSuccess ? e : cudaErrorInvalidDevice);
+        return AVE_ERR_CUDA;
+    }
+    void *scratch = scratch_of_device[dev].load(std::memory_order_acquire);
+    if (!scratch) {
+        e = cudaGetSymbolAddress(&scratch, g_splitkv_static_scratch);
+        if (e != cudaSuccess || !scratch) {
+            t_last_cuda_error = int(e);
+            return AVE_ERR_CUDA;
+        }
+        scratch_of_device[dev].store(scratch, std::memory_order_release);
+    }
+    const size_t rows = size_t(B) * H * Sq;
+    float *o_partial = static_cast<float *>(scratch);
+    float *lse_partial = o_partial + size_t(n_splits) * rows * D;
+    return run_splitkv(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, causal, scale, n_splits, o_partial, lse_partial,
+                       static_cast<cudaStream_t>(stream));
+}
+
 int ave_attn_device_status(unsigned int *raw_word) {
     cudaError_t e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
@@ -368,6 +411,8 @@ const char *ave_attn_strerror(int status) {
         case AVE_ERR_CUDA: return "a CUDA call failed (see ave_attn_last_cuda_error)";
         case AVE_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel gave up";
         case AVE_ERR_WORKSPACE: return "workspace is NULL, misaligned or too small";
+        case AVE_ERR_STATIC_SCRATCH:
+            return "the problem needs more scratch than the built-in array of ave_attn_fwd_splitkv_static holds";
         default: return "unknown status";
     }
 }
