@@ -28,6 +28,9 @@ METRIC = "attention fwd TFLOP/s (bf16, causal=half FLOPs)"
 UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "c2_mha_prefill"
 NOMINAL_BF16_TFLOPS = 2250.0          # vendor dense bf16 figure, context only
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu captures summarised under
+# profiles/ (attn_fwd_ws_<workload>_ncu_full.md); null for workloads that were not captured.
+NCU_DRAM_BYTES_PER_LAUNCH = {"c2_mha_prefill": 320.5e6, "c3_gqa_prefill": 271.8e6}
 FALLBACK_BF16_TFLOPS = 1590.0         # earlier measurement on this machine, used when no measured file exists
 
 
@@ -272,7 +275,9 @@ def run_ours(args):
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
             "gpu_launches": int(launches),
             "roofline": {"bound": "tensor", "achieved": kernel_tf, "peak": peak, "unit": "TFLOP/s",
-                         "frac": kernel_tf / peak, "traffic": None, "peak_kind": peak_kind,
+                         "frac": kernel_tf / peak, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(w.name),
+                         "traffic_unit": "bytes per launch (ncu dram read+write)",
+                         "algorithmic_hbm_bytes": inputs.min_hbm_bytes(w), "peak_kind": peak_kind,
                          "frac_of_nominal_2250": kernel_tf / NOMINAL_BF16_TFLOPS,
                          "flops_per_launch": flops, "kernel_us": 1e3 * ms / args.steps},
         }
