@@ -43,6 +43,7 @@ struct FwdParams {
     // BN); a work tile handles one range and writes a normalised fp32 partial result.
     int n_splits;
     int keys_per_split;
+    int rows_per_head;   // > 0: rows are (query head in group, query position) pairs, this many positions per head
     float *o_partial;    // fp32 [n_splits, B*H, Sq, D]
     float *lse_partial;  // fp32 [n_splits, B*H, Sq]
 };

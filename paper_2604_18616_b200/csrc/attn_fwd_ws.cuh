@@ -93,11 +93,27 @@ struct WorkTileT<true> : WorkTileBase {
     int split;           // index of the key range
 };
 
-// Number of key tiles a 128-row sub-tile starting at row i0 must visit inside [k_begin, k_end).
+// Split-KV launches may pack the G query heads of a key/value head into the rows of one problem
+// ("head" = KV head, row r = head_in_group * rows_per_head + query position): the rows of Q, O and LSE
+// are contiguous that way, and only the causal mask needs the query position r % rows_per_head.
+// Smallest and one-past-largest query position among the rows [i0, i0 + BM):
+__device__ __forceinline__ int query_pos_lo(int i0, int rows_per_head) {
+    if (rows_per_head <= 0) return i0;
+    const int lo = i0 % rows_per_head;
+    return (lo + BM > rows_per_head) ? 0 : lo;
+}
+__device__ __forceinline__ int query_pos_hi(int i0, int rows_per_head) {
+    if (rows_per_head <= 0) return i0 + BM;
+    const int lo = i0 % rows_per_head;
+    return (lo + BM >= rows_per_head) ? rows_per_head : lo + BM;
+}
+
+// Number of key tiles a 128-row sub-tile must visit inside [k_begin, k_end); pos_hi is one past the
+// largest query position among its rows.
 template <bool CAUSAL>
-__device__ __forceinline__ int kv_tiles_for(int i0, int causal_off, int k_begin, int k_end) {
+__device__ __forceinline__ int kv_tiles_for(int pos_hi, int causal_off, int k_begin, int k_end) {
     int hi = k_end;
-    if (CAUSAL) hi = min(hi, i0 + BM + causal_off);  // one past the last key the sub-tile's last row may see
+    if (CAUSAL) hi = min(hi, pos_hi + causal_off);  // one past the last key any row of the sub-tile may see
     return hi > k_begin ? (hi - k_begin + BN - 1) / BN : 0;
 }
 
@@ -140,8 +156,8 @@ __device__ __forceinline__ WorkTileT<SPLIT> decode_tile(int id, const FwdParams 
     w.bg = b * p.Hkv + h / (p.H / p.Hkv);
     w.q0 = qb * 2 * BM;
     if constexpr (SPLIT) {
-        w.n0 = kv_tiles_for<CAUSAL>(w.q0, p.causal_off, k_begin, k_end);
-        w.n1 = kv_tiles_for<CAUSAL>(w.q0 + BM, p.causal_off, k_begin, k_end);
+        w.n0 = kv_tiles_for<CAUSAL>(query_pos_hi(w.q0, p.rows_per_head), p.causal_off, k_begin, k_end);
+        w.n1 = max(w.n0, kv_tiles_for<CAUSAL>(query_pos_hi(w.q0 + BM, p.rows_per_head), p.causal_off, k_begin, k_end));
     } else {
         w.n0 = kv_tiles_whole<CAUSAL>(w.q0, p.Sq, p.Sk);
         w.n1 = kv_tiles_whole<CAUSAL>(w.q0 + BM, p.Sq, p.Sk);
@@ -564,8 +580,16 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     const int k_end = key_end(w, p);
                     const int j0 = key_begin(w) + j * BN;  // first key of this step
                     int lim = k_end - 1 - j0;           // columns c <= lim of this tile are visible to row i
-                    if (CAUSAL) lim = min(lim, i + off - j0);
-                    const bool need_mask = (j0 + BN > k_end) || (CAUSAL && (j0 + BN - 1 > i0 + off));
+                    bool need_mask;
+                    if constexpr (SPLIT) {
+                        const int pos = p.rows_per_head > 0 ? i % p.rows_per_head : i;  // query position of row i
+                        if (CAUSAL) lim = min(lim, pos + off - j0);
+                        need_mask = (j0 + BN > k_end) ||
+                                    (CAUSAL && (j0 + BN - 1 > query_pos_lo(i0, p.rows_per_head) + off));
+                    } else {
+                        if (CAUSAL) lim = min(lim, i + off - j0);
+                        need_mask = (j0 + BN > k_end) || (CAUSAL && (j0 + BN - 1 > i0 + off));
+                    }
 
                     // ---- row extreme of the raw scores (maximum of scale*s is at max s, or min s if scale < 0)
                     // With a positive scale a masked score is simply replaced by -inf: it then drops out

@@ -140,7 +140,7 @@ int launch_ws(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &t
 // and writes fp32 partials.
 int launch_attention(const void *q, const void *k, const void *v, void *o, float *lse, int B, int H, int Hkv, int Sq,
                      int Sk, int D, int causal, float scale, int n_splits, int keys_per_split, float *o_partial,
-                     float *lse_partial, cudaStream_t s) {
+                     float *lse_partial, int rows_per_head, cudaStream_t s) {
     CUtensorMap tq, tk, tv, to;
     if (!encode_map(&tq, q, D, Sq, (long long)B * H, ave::BM)) return AVE_ERR_CUDA;
     if (!encode_map(&to, o, D, Sq, (long long)B * H, ave::WsCfg<128>::kOutBoxRows)) return AVE_ERR_CUDA;
@@ -157,7 +157,8 @@ int launch_attention(const void *q, const void *k, const void *v, void *o, float
     p.Sk = Sk;
     p.BH = B * H;
     p.n_qblk = (Sq + 2 * ave::BM - 1) / (2 * ave::BM);
-    p.causal_off = Sk - Sq;
+    p.causal_off = Sk - (rows_per_head > 0 ? rows_per_head : Sq);
+    p.rows_per_head = rows_per_head;
     p.n_splits = split ? n_splits : 1;
     p.keys_per_split = split ? keys_per_split : Sk;
     p.o_partial = o_partial;
@@ -234,8 +235,15 @@ int run_splitkv(const void *q, const void *k, const void *v, void *o, float *lse
                 int Sk, int D, int causal, float scale, int n_splits, float *o_partial, float *lse_partial,
                 cudaStream_t s) {
     const int kps = splitkv_keys_per_split(Sk, n_splits);
-    int st = launch_attention(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, causal, scale, n_splits, kps, o_partial,
-                              lse_partial, s);
+    // With grouped-query heads and few query rows, the G query heads of a KV head become rows of one
+    // problem with Hkv heads of G * Sq rows each: Q, O, LSE and the partials are laid out exactly the
+    // same in memory, and one work tile then serves up to 256 / Sq query heads per pass over K/V.
+    const int G = H / Hkv;
+    const bool pack = G > 1 && Sq < 2 * ave::BM && (long long)G * Sq < (1ll << 30);
+    int st = pack ? launch_attention(q, k, v, o, lse, B, Hkv, Hkv, G * Sq, Sk, D, causal, scale, n_splits, kps,
+                                     o_partial, lse_partial, Sq, s)
+                  : launch_attention(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, causal, scale, n_splits, kps, o_partial,
+                                     lse_partial, 0, s);
     if (st != AVE_OK) return st;
     const long long rows = (long long)B * H * Sq;
     const long long work = rows * (D / 8);
@@ -263,7 +271,7 @@ int ave_attn_fwd(const void *q, const void *k, const void *v, void *o, float *ls
     if (st != AVE_OK) return st;
     st = check_device();
     if (st != AVE_OK) return st;
-    return launch_attention(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, causal, scale, 1, 0, nullptr, nullptr,
+    return launch_attention(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, causal, scale, 1, 0, nullptr, nullptr, 0,
                             static_cast<cudaStream_t>(stream));
 }
 

@@ -88,3 +88,34 @@ def test_splitkv_argument_checks():
     with pytest.raises(binding.AveAttnError) as e:
         binding.ave_attn_fwd_splitkv(q, kv, kv, 0, workspace=small)
     assert e.value.status == binding.AVE_ERR_BAD_SHAPE
+
+
+PACKED = [
+    # grouped-query heads with few query rows: the G heads of a KV head share work tiles
+    (2, 16, 2, 1, 3000, 128, True, 4),
+    (1, 8, 1, 37, 700, 64, True, 2),      # 8 * 37 = 296 rows: tiles straddle heads, causal positions wrap
+    (1, 12, 4, 100, 1000, 128, True, 3),  # G = 3
+    (2, 8, 2, 255, 600, 128, True, 2),
+    (1, 16, 4, 5, 2048, 128, False, 8),
+]
+
+
+@pytest.mark.parametrize("B,H,Hkv,Sq,Sk,D,causal,n_splits", PACKED)
+def test_splitkv_packed_query_heads(B, H, Hkv, Sq, Sk, D, causal, n_splits):
+    q, k, v = rand_qkv(Sq + Sk * 3 + H, B, H, Hkv, Sq, Sk, D)
+    scale = 1.0 / math.sqrt(D)
+    o, lse = run_split(q, k, v, causal, scale, n_splits)
+    o_ref, lse_ref = oracle.attn_fwd(q, k, v, causal, scale)
+    parity.compare(o, lse, o_ref, lse_ref, "packed %s" % ((B, H, Hkv, Sq, Sk, D, causal, n_splits),))
+
+
+def test_splitkv_packed_heads_read_their_own_kv_head():
+    # per-KV-head constant V: every query head must return its own group's constant
+    B, H, Hkv, Sq, Sk, D = 1, 8, 4, 3, 500, 64
+    q, k, _ = rand_qkv(5, B, H, Hkv, Sq, Sk, D)
+    v = torch.zeros(B, Hkv, Sk, D, dtype=torch.bfloat16)
+    for g in range(Hkv):
+        v[:, g] = float(g + 1)
+    o, _ = run_split(q, k, v, True, 0.125, 2)
+    for h in range(H):
+        assert torch.all(o[:, h] == float(h // 2 + 1))
