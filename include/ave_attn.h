@@ -67,6 +67,29 @@ int ave_attn_fwd(const void *q, const void *k, const void *v, void *o, float *ls
                  int causal, float scale, void *stream);
 
 /*
+ * The same operation for tensors that are not contiguous [B, heads, rows, D]
+ * arrays: each of q, k, v, o is described by its base DEVICE pointer and three
+ * strides, in ELEMENTS (bf16), of its batch, head and row dimensions, in that
+ * order; the D elements of a row are contiguous.  Element (b, h, i, d) of q is
+ * at q + b*q_strides[0] + h*q_strides[1] + i*q_strides[2] + d, likewise for
+ * k, v (heads = Hkv, rows = Sk) and o.  This covers the paper's Fig. 1 layout
+ * (sequence, head, d) -- strides {S*H*D, D, H*D} -- and a packed [B, S, 3, H, D]
+ * QKV buffer -- base pointers D*H elements apart, strides {3*S*H*D, D, 3*H*D} --
+ * without copies.  lse stays a contiguous fp32 [B, H, Sq] array.
+ * Every stride must be positive, a multiple of 8 elements (16 bytes) and below
+ * 2^38; a row stride must be at least D.  The strides of o must not make two
+ * of its rows overlap (not checked).  The stride arrays are HOST pointers, read
+ * before the call returns.  Everything else as for ave_attn_fwd; a NULL stride
+ * array is AVE_ERR_NULL_POINTER, a non-positive or too large stride
+ * AVE_ERR_BAD_SHAPE, a stride that is not a multiple of 8 AVE_ERR_MISALIGNED.
+ */
+int ave_attn_fwd_strided(const void *q, const void *k, const void *v, void *o, float *lse,
+                         int B, int H, int Hkv, int Sq, int Sk, int D,
+                         const long long *q_strides, const long long *k_strides,
+                         const long long *v_strides, const long long *o_strides,
+                         int causal, float scale, void *stream);
+
+/*
  * The same operation for tensors that live in HOST memory (same layouts and
  * limits).  The call enqueues, on `stream`: host-to-device copies of q, k, v
  * into `workspace`, the attention kernel, and device-to-host copies of o and

@@ -49,6 +49,8 @@ def lib() -> ctypes.CDLL:
         vp, ci, cf = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
         L.ave_attn_fwd.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, cf, vp]
         L.ave_attn_fwd.restype = ci
+        L.ave_attn_fwd_strided.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, vp, vp, vp, vp, ci, cf, vp]
+        L.ave_attn_fwd_strided.restype = ci
         L.ave_attn_fwd_host.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, cf, vp, ctypes.c_size_t, vp]
         L.ave_attn_fwd_host.restype = ci
         L.ave_attn_host_workspace_bytes.argtypes = [ci] * 6
@@ -137,6 +139,34 @@ def ave_attn_fwd(q, k, v, o=None, lse=None, causal=False, scale=None, stream=Non
             B, H, Hkv, Sq, Sk, D, int(bool(causal)), float(scale), _stream_ptr(stream))
     if st != AVE_OK:
         raise AveAttnError(st, "ave_attn_fwd")
+    return o, lse
+
+
+def ave_attn_fwd_strided(q, k, v, o, lse=None, causal=False, scale=None, stream=None):
+    """The same for strided views: q, o are [B,H,Sq,D] and k, v [B,Hkv,Sk,D] CUDA bf16 tensors with any
+    batch/head/row strides (last dimension contiguous), e.g. permuted views of (B,S,H,D) storage or slices
+    of a packed QKV buffer; ``o`` is written in place through its strides.  ``lse`` is contiguous fp32."""
+    for t in (q, k, v, o):
+        if not (t.is_cuda and t.dtype == torch.bfloat16 and t.dim() == 4 and t.stride(3) == 1):
+            raise ValueError("q, k, v, o must be 4-D CUDA bfloat16 tensors whose last dimension is contiguous")
+    B, H, Sq, D = q.shape
+    Bk, Hkv, Sk, Dk = k.shape
+    if tuple(v.shape) != tuple(k.shape) or Bk != B or Dk != D or tuple(o.shape) != tuple(q.shape):
+        raise ValueError("inconsistent q/k/v/o shapes")
+    if lse is None:
+        lse = torch.empty((B, H, Sq), dtype=torch.float32, device=q.device)
+    if scale is None:
+        scale = D ** -0.5
+    arrs = [(ctypes.c_longlong * 3)(t.stride(0), t.stride(1), t.stride(2)) for t in (q, k, v, o)]
+    with torch.cuda.device(q.device):
+        st = lib().ave_attn_fwd_strided(
+            ctypes.c_void_p(q.data_ptr()), ctypes.c_void_p(k.data_ptr()), ctypes.c_void_p(v.data_ptr()),
+            ctypes.c_void_p(o.data_ptr()), ctypes.c_void_p(lse.data_ptr()),
+            B, H, Hkv, Sq, Sk, D, ctypes.cast(arrs[0], ctypes.c_void_p), ctypes.cast(arrs[1], ctypes.c_void_p),
+            ctypes.cast(arrs[2], ctypes.c_void_p), ctypes.cast(arrs[3], ctypes.c_void_p),
+            int(bool(causal)), float(scale), _stream_ptr(stream))
+    if st != AVE_OK:
+        raise AveAttnError(st, "ave_attn_fwd_strided")
     return o, lse
 
 

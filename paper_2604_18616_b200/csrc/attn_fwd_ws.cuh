@@ -81,7 +81,8 @@ __device__ __forceinline__ void setmaxnreg_dec() {
 // One work tile, decoded from its position in the launch order.
 struct WorkTileBase {
     int bh;      // b * H + h
-    int bg;      // b * Hkv + h / (H / Hkv): key/value head (Fig. 1: idx_h / gqa)
+    int b, h;    // batch and query head
+    int g;       // h / (H / Hkv): key/value head (Fig. 1: idx_h / gqa)
     int q0;      // first query row
     int n0, n1;  // key tiles the two sub-tiles visit (n1 >= n0)
 };
@@ -151,9 +152,9 @@ __device__ __forceinline__ WorkTileT<SPLIT> decode_tile(int id, const FwdParams 
     const int rank = rem / hg;
     w.bh = bh0 + (rem - rank * hg);
     const int qb = CAUSAL ? (p.n_qblk - 1 - rank) : rank;
-    const int b = w.bh / p.H;
-    const int h = w.bh - b * p.H;
-    w.bg = b * p.Hkv + h / (p.H / p.Hkv);
+    w.b = w.bh / p.H;
+    w.h = w.bh - w.b * p.H;
+    w.g = w.h / (p.H / p.Hkv);
     w.q0 = qb * 2 * BM;
     if constexpr (SPLIT) {
         w.n0 = kv_tiles_for<CAUSAL>(query_pos_hi(w.q0, p.rows_per_head), p.causal_off, k_begin, k_end);
@@ -328,9 +329,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     if (leader) {
                         const uint32_t bar = smem_u32(&bar_q_full[t]);
                         mbar_arrive_expect_tx(bar, Cfg::kTileBytes);
-                        for (int x = 0; x < Cfg::kBoxes; ++x)
-                            tma_load_3d(sQ + t * Cfg::kTileBytes + x * Cfg::kBoxBytes, &tm_q, bar, x * 64,
-                                        w.q0 + t * BM, w.bh);
+                        for (int x = 0; x < Cfg::kBoxes; ++x)  // the tensor maps are {D, rows, heads, batch}
+                            tma_load_4d(sQ + t * Cfg::kTileBytes + x * Cfg::kBoxBytes, &tm_q, bar, x * 64,
+                                        w.q0 + t * BM, w.h, w.b);
                     }
                 };
                 try_load_q(0, false);
@@ -368,8 +369,8 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         if (n == kTraceTile) trace_stamp(3, it >> 1, it & 1);
                         mbar_arrive_expect_tx(bar, Cfg::kTileBytes);
                         for (int x = 0; x < Cfg::kBoxes; ++x)
-                            tma_load_3d(sRing + slot * Cfg::kTileBytes + x * Cfg::kBoxBytes, tm, bar, x * 64,
-                                        key_begin(w) + (it >> 1) * BN, w.bg);
+                            tma_load_4d(sRing + slot * Cfg::kTileBytes + x * Cfg::kBoxBytes, tm, bar, x * 64,
+                                        key_begin(w) + (it >> 1) * BN, w.g, w.b);
                     }
                 }
                 if (ok) try_load_q(0, true);
@@ -780,7 +781,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         fence_proxy_async_smem();
                         __syncwarp();
                         if (lane == 0 && i0 + wq * 32 < p.Sq) {
-                            tma_store_3d(&tm_o, sO, x * 64, i0 + wq * 32, bh);
+                            tma_store_4d(&tm_o, sO, x * 64, i0 + wq * 32, w.h, w.b);
                             tma_store_commit();
                             store_pending = true;
                         }

@@ -48,16 +48,25 @@ EncodeTiledFn encode_fn() {
     return f;
 }
 
-// bf16 tensor [n_mat, rows, D] (D contiguous) as a 3-D map with a box of
-// 64 columns x box_rows rows, 128-byte swizzle, zero fill outside the tensor.
-bool encode_map(CUtensorMap *map, const void *base, int D, int rows, long long n_mat, int box_rows) {
+// Element strides of one tensor's batch, head and row dimensions (the D elements of a row are contiguous).
+struct Strides {
+    long long batch, head, row;
+};
+Strides contiguous_strides(int heads, int rows, int D) {
+    return Strides{(long long)heads * rows * D, (long long)rows * D, (long long)D};
+}
+
+// bf16 tensor [batch, heads, rows, D] with the given strides as a 4-D map {D, rows, heads, batch} with a
+// box of 64 columns x box_rows rows, 128-byte swizzle, zero fill outside the tensor.
+bool encode_map(CUtensorMap *map, const void *base, int D, int rows, int heads, int batch, const Strides &st,
+                int box_rows) {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return false;
-    cuuint64_t gdim[3] = {cuuint64_t(D), cuuint64_t(rows), cuuint64_t(n_mat)};
-    cuuint64_t gstride[2] = {cuuint64_t(D) * 2, cuuint64_t(rows) * cuuint64_t(D) * 2};
-    cuuint32_t box[3] = {64, cuuint32_t(box_rows), 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), gdim, gstride, box, estr,
+    cuuint64_t gdim[4] = {cuuint64_t(D), cuuint64_t(rows), cuuint64_t(heads), cuuint64_t(batch)};
+    cuuint64_t gstride[3] = {cuuint64_t(st.row) * 2, cuuint64_t(st.head) * 2, cuuint64_t(st.batch) * 2};
+    cuuint32_t box[4] = {64, cuuint32_t(box_rows), 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), gdim, gstride, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -138,14 +147,19 @@ int launch_ws(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &t
 // Encode the tensor maps, fill the kernel parameters and launch.  n_splits == 1 with no partial
 // buffers is the ordinary forward; otherwise every work tile covers one range of keys_per_split keys
 // and writes fp32 partials.
+// `layout` (strides of q, k, v, o in this order) is NULL for contiguous [B, heads, rows, D] tensors.
 int launch_attention(const void *q, const void *k, const void *v, void *o, float *lse, int B, int H, int Hkv, int Sq,
                      int Sk, int D, int causal, float scale, int n_splits, int keys_per_split, float *o_partial,
-                     float *lse_partial, int rows_per_head, cudaStream_t s) {
+                     float *lse_partial, int rows_per_head, const Strides *layout, cudaStream_t s) {
+    const Strides sq = layout ? layout[0] : contiguous_strides(H, Sq, D);
+    const Strides sk = layout ? layout[1] : contiguous_strides(Hkv, Sk, D);
+    const Strides sv = layout ? layout[2] : contiguous_strides(Hkv, Sk, D);
+    const Strides so = layout ? layout[3] : contiguous_strides(H, Sq, D);
     CUtensorMap tq, tk, tv, to;
-    if (!encode_map(&tq, q, D, Sq, (long long)B * H, ave::BM)) return AVE_ERR_CUDA;
-    if (!encode_map(&to, o, D, Sq, (long long)B * H, ave::WsCfg<128>::kOutBoxRows)) return AVE_ERR_CUDA;
-    if (!encode_map(&tk, k, D, Sk, (long long)B * Hkv, ave::BN)) return AVE_ERR_CUDA;
-    if (!encode_map(&tv, v, D, Sk, (long long)B * Hkv, ave::BN)) return AVE_ERR_CUDA;
+    if (!encode_map(&tq, q, D, Sq, H, B, sq, ave::BM)) return AVE_ERR_CUDA;
+    if (!encode_map(&to, o, D, Sq, H, B, so, ave::WsCfg<128>::kOutBoxRows)) return AVE_ERR_CUDA;
+    if (!encode_map(&tk, k, D, Sk, Hkv, B, sk, ave::BN)) return AVE_ERR_CUDA;
+    if (!encode_map(&tv, v, D, Sk, Hkv, B, sv, ave::BN)) return AVE_ERR_CUDA;
 
     const bool split = o_partial != nullptr;
     ave::FwdParams p;
@@ -241,9 +255,9 @@ int run_splitkv(const void *q, const void *k, const void *v, void *o, float *lse
     const int G = H / Hkv;
     const bool pack = G > 1 && Sq < 2 * ave::BM && (long long)G * Sq < (1ll << 30);
     int st = pack ? launch_attention(q, k, v, o, lse, B, Hkv, Hkv, G * Sq, Sk, D, causal, scale, n_splits, kps,
-                                     o_partial, lse_partial, Sq, s)
+                                     o_partial, lse_partial, Sq, nullptr, s)
                   : launch_attention(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, causal, scale, n_splits, kps, o_partial,
-                                     lse_partial, 0, s);
+                                     lse_partial, 0, nullptr, s);
     if (st != AVE_OK) return st;
     const long long rows = (long long)B * H * Sq;
     const long long work = rows * (D / 8);
@@ -271,7 +285,32 @@ int ave_attn_fwd(const void *q, const void *k, const void *v, void *o, float *ls
     if (st != AVE_OK) return st;
     st = check_device();
     if (st != AVE_OK) return st;
-    return launch_attention(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, causal, scale, 1, 0, nullptr, nullptr, 0,
+    return launch_attention(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, causal, scale, 1, 0, nullptr, nullptr, 0, nullptr,
+                            static_cast<cudaStream_t>(stream));
+}
+
+int ave_attn_fwd_strided(const void *q, const void *k, const void *v, void *o, float *lse, int B, int H, int Hkv,
+                         int Sq, int Sk, int D, const long long *q_strides, const long long *k_strides,
+                         const long long *v_strides, const long long *o_strides, int causal, float scale,
+                         void *stream) {
+    if (!q_strides || !k_strides || !v_strides || !o_strides) return AVE_ERR_NULL_POINTER;
+    int st = validate(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, scale);
+    if (st >= 0) return st;
+    Strides layout[4];
+    const long long *in[4] = {q_strides, k_strides, v_strides, o_strides};
+    for (int i = 0; i < 4; ++i) {
+        layout[i] = Strides{in[i][0], in[i][1], in[i][2]};
+        if (layout[i].batch <= 0 || layout[i].head <= 0 || layout[i].row < D) return AVE_ERR_BAD_SHAPE;
+        if (layout[i].batch >= (1ll << 38) || layout[i].head >= (1ll << 38) || layout[i].row >= (1ll << 38))
+            return AVE_ERR_BAD_SHAPE;  // the tensor map holds byte strides below 2^40
+    }
+    for (int i = 0; i < 4; ++i)
+        if ((layout[i].batch | layout[i].head | layout[i].row) & 7) return AVE_ERR_MISALIGNED;  // 16-byte units
+    st = validate_ptrs_and_scale(q, k, v, o, lse, scale);
+    if (st != AVE_OK) return st;
+    st = check_device();
+    if (st != AVE_OK) return st;
+    return launch_attention(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, causal, scale, 1, 0, nullptr, nullptr, 0, layout,
                             static_cast<cudaStream_t>(stream));
 }
 

@@ -76,21 +76,21 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
 __device__ __forceinline__ void tma_prefetch_desc(const void *tmap) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");
 }
-// 3-D tiled load, global -> shared, completion counted in bytes on `bar`.
+// 4-D tiled load, global -> shared, completion counted in bytes on `bar`.
 // x (innermost coordinate) must keep x * sizeof(element) a multiple of 16.
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const void *tmap, uint32_t bar,
-                                            int x, int y, int z) {
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const void *tmap, uint32_t bar,
+                                            int x, int y, int z, int w) {
     asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
-        "[%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar), "r"(x), "r"(y), "r"(z)
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar), "r"(x), "r"(y), "r"(z), "r"(w)
         : "memory");
 }
-// 3-D tiled store, shared -> global (rows outside the tensor are clipped).
-__device__ __forceinline__ void tma_store_3d(const void *tmap, uint32_t src, int x, int y, int z) {
+// 4-D tiled store, shared -> global (rows outside the tensor are clipped).
+__device__ __forceinline__ void tma_store_4d(const void *tmap, uint32_t src, int x, int y, int z, int w) {
     asm volatile(
-        "cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
-        ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(src), "r"(x), "r"(y), "r"(z)
+        "cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+        ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(src), "r"(x), "r"(y), "r"(z), "r"(w)
         : "memory");
 }
 __device__ __forceinline__ void tma_store_commit() {
