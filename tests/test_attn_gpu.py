@@ -61,6 +61,26 @@ def test_small_and_ragged_shapes(B, H, Hkv, Sq, Sk, D, causal):
     parity.check_full(q, k, v, causal, 1.0 / math.sqrt(D), "shape %s" % ((B, H, Hkv, Sq, Sk, D, causal),))
 
 
+def _random_shapes(n, seed):
+    """Seeded random problem shapes: sizes on and around tile edges, every head grouping, both D."""
+    rng = np.random.default_rng(seed)
+    out = []
+    for _ in range(n):
+        hkv = int(rng.choice([1, 2, 3]))
+        g = int(rng.choice([1, 2, 4]))
+        edge = lambda: int(rng.choice([1, 64, 127, 128, 129, 255, 256, 257, 383, 512]) + rng.integers(0, 3))
+        sq, sk = (edge(), edge()) if rng.random() < 0.7 else (int(rng.integers(1, 700)), int(rng.integers(1, 900)))
+        out.append((int(rng.integers(1, 3)), hkv * g, hkv, sq, sk, int(rng.choice([64, 128])), bool(rng.random() < 0.6),
+                    float(rng.choice([0.05, 0.088, 0.125, 0.3]))))
+    return out
+
+
+@pytest.mark.parametrize("B,H,Hkv,Sq,Sk,D,causal,scale", _random_shapes(24, 2024))
+def test_seeded_random_shapes(B, H, Hkv, Sq, Sk, D, causal, scale):
+    q, k, v = rand_qkv(Sq * 1009 + Sk, B, H, Hkv, Sq, Sk, D)
+    parity.check_full(q, k, v, causal, scale, "random shape %s" % ((B, H, Hkv, Sq, Sk, D, causal, scale),))
+
+
 @pytest.mark.parametrize("scale", [0.0, -0.1, 0.02, 0.3])
 @pytest.mark.parametrize("causal", [False, True])
 def test_scale_values_including_zero_and_negative(scale, causal):
@@ -160,6 +180,7 @@ def test_errors_launch_nothing_and_leave_outputs_alone():
     ("c3_gqa_prefill", 1024),
     ("c4_long_context", 768),
     ("c5_wide_noncausal", 768),
+    ("paper_gqa_n2048", 512),       # the paper's own evaluation shape (one KV head shared by 8 query heads)
 ])
 def test_full_size_configs_sampled_rows(name, n_random):
     w = inputs.get(name)
