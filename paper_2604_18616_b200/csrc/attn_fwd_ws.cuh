@@ -22,6 +22,8 @@
 // whole score row in registers.
 #pragma once
 
+#include <type_traits>
+
 #include "attn_common.cuh"
 #include "softmax_math.cuh"
 
@@ -565,10 +567,23 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 if (lane == 0) mbar_arrive(smem_u32(&bar_o_free[t]));
             } else {
                 float m_run = -INFINITY, l_run = 0.f;
-                for (int j = 0; j < n_t; ++j) {
+                // Steps [0, n_full) lie wholly below the causal diagonal and inside the key range: nothing
+                // to mask.  The step is instantiated twice, with and without the masking code, and the
+                // choice is made once per tile here: left as a run-time flag inside one body, the
+                // per-element compares and selects end up predicated into every step.
+                const int k_end = key_end(w, p);
+                int n_full = (k_end - key_begin(w)) / BN;
+                if (CAUSAL) {
+                    const int pos_lo = SPLIT ? query_pos_lo(i0, p.rows_per_head) : i0;
+                    const int num = pos_lo + off - key_begin(w) + 1;  // keys every row of the sub-tile sees
+                    n_full = min(n_full, num > 0 ? num / BN : 0);
+                }
+                n_full = max(0, min(n_full, n_t));
+                auto step = [&](const int j, auto masked_tag) -> bool {
+                    constexpr bool need_mask = decltype(masked_tag)::value;
                     if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 0);
                     ok = wait_bar(&bar_s[t], ns & 1, STATUS_TIMEOUT_MMA);
-                    if (!ok) break;
+                    if (!ok) return false;
                     ++ns;
                     if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 1);
                     tc_fence_after();
@@ -578,18 +593,13 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     tmem_wait_ld();
                     if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 2);
 
-                    const int k_end = key_end(w, p);
                     const int j0 = key_begin(w) + j * BN;  // first key of this step
                     int lim = k_end - 1 - j0;           // columns c <= lim of this tile are visible to row i
-                    bool need_mask;
                     if constexpr (SPLIT) {
                         const int pos = p.rows_per_head > 0 ? i % p.rows_per_head : i;  // query position of row i
                         if (CAUSAL) lim = min(lim, pos + off - j0);
-                        need_mask = (j0 + BN > k_end) ||
-                                    (CAUSAL && (j0 + BN - 1 > query_pos_lo(i0, p.rows_per_head) + off));
                     } else {
                         if (CAUSAL) lim = min(lim, i + off - j0);
-                        need_mask = (j0 + BN > k_end) || (CAUSAL && (j0 + BN - 1 > i0 + off));
                     }
 
                     // ---- row extreme of the raw scores (maximum of scale*s is at max s, or min s if scale < 0)
@@ -719,6 +729,14 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&bar_p[t]));
                     if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 5);
+                    return true;
+                };
+                {
+                    int j = 0;
+                    for (; j < n_full; ++j)
+                        if (!step(j, std::false_type{})) break;
+                    for (; ok && j < n_t; ++j)
+                        if (!step(j, std::true_type{})) break;
                 }
 
                 // ---- epilogue: O / l -> bf16 -> shared (TMA layout) -> global; LSE = ln2 * (m + log2 l)
