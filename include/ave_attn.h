@@ -36,7 +36,7 @@ typedef enum {
     AVE_OK = 0,
     AVE_ERR_NULL_POINTER = 1,       /* q, k, v, o or lse is NULL */
     AVE_ERR_BAD_SHAPE = 2,          /* a size <= 0, H % Hkv != 0, or a size beyond the limits below */
-    AVE_ERR_UNSUPPORTED_D = 3,      /* D not in {64, 128} */
+    AVE_ERR_UNSUPPORTED_D = 3,      /* D not a multiple of 8 in [8, 128] (split-KV calls: not 64 or 128) */
     AVE_ERR_MISALIGNED = 4,         /* q, k, v, o not 16-byte aligned, or lse not 4-byte aligned */
     AVE_ERR_BAD_SCALE = 5,          /* scale is NaN or infinite (zero and negative values are allowed) */
     AVE_ERR_UNSUPPORTED_DEVICE = 6, /* the current device is not compute capability 10.x */
@@ -54,7 +54,10 @@ typedef enum {
  *   v   bf16 [B, Hkv, Sk, D]   read
  *   o   bf16 [B, H,   Sq, D]   written
  *   lse fp32 [B, H,   Sq]      written
- * Limits: D in {64, 128}; H % Hkv == 0; Sq, Sk < 2^31 / 2; B * H < 2^31.
+ * Limits: D a multiple of 8, 8 <= D <= 128 (the kernels compute with D rounded
+ * up to 64 or 128: the loads zero-fill the extra columns, the stores clip them,
+ * so D = 96 costs what D = 128 costs); H % Hkv == 0; Sq, Sk < 2^31 / 2;
+ * B * H < 2^31.
  * causal: 0 = every key visible, nonzero = bottom-right aligned causal mask.
  * scale: multiplies Q K^T before the softmax (callers normally pass 1/sqrt(D)).
  * stream: a cudaStream_t; NULL is the legacy default stream.
@@ -115,7 +118,8 @@ size_t ave_attn_host_workspace_bytes(int B, int H, int Hkv, int Sq, int Sk, int 
  *   LSE = ln sum_s exp(LSE_s),   O = sum_s exp(LSE_s - LSE) * O_s,
  * which is the same re-association of the softmax sum that the tiling of paper
  * Section 2 relies on, applied across CTAs.  Same tensors, layouts, limits and
- * result as ave_attn_fwd (up to rounding order); meant for few query rows
+ * result as ave_attn_fwd (up to rounding order), except that D must be 64 or
+ * 128; meant for few query rows
  * against many keys (decode, chunked prefill), where one work tile per
  * (batch, head, 256 query rows) would leave most SMs idle.
  * n_splits: 1 .. AVE_SPLITKV_MAX_SPLITS; each range is ceil(Sk / n_splits)

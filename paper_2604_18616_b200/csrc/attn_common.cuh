@@ -29,8 +29,10 @@ constexpr long long WAIT_LIMIT_CYCLES = 1ll << 29;
 constexpr uint32_t WAIT_LIMIT = 1u << 16;
 
 struct FwdParams {
-    void *o;          // bf16 [B, H, Sq, D]
+    void *o;          // bf16 [B, H, Sq, D] through the strides below
     float *lse;       // fp32 [B, H, Sq]
+    long long o_stride_b, o_stride_h, o_stride_r;  // element strides of o (rows written without TMA use them)
+    int d_true;       // head dimension of the tensors (<= the kernel's D; TMA zero-fills / clips the rest)
     int H, Hkv;       // query heads, key/value heads
     int Sq, Sk;       // sequence lengths
     int BH;           // B * H

@@ -557,8 +557,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         for (int c = 0; c < D / 4; ++c) reinterpret_cast<uint4 *>(p.o_partial + row * D)[c] = z;
                         p.lse_partial[row] = -INFINITY;
                     } else {
-                        __nv_bfloat16 *o_row = reinterpret_cast<__nv_bfloat16 *>(p.o) + (size_t(bh) * p.Sq + i) * D;
-                        for (int c = 0; c < D / 8; ++c) reinterpret_cast<uint4 *>(o_row)[c] = z;
+                        __nv_bfloat16 *o_row = reinterpret_cast<__nv_bfloat16 *>(p.o) + w.b * p.o_stride_b +
+                                               w.h * p.o_stride_h + i * p.o_stride_r;
+                        for (int c = 0; c < p.d_true / 8; ++c) reinterpret_cast<uint4 *>(o_row)[c] = z;
                         p.lse[size_t(bh) * p.Sq + i] = -INFINITY;
                     }
                 }

@@ -83,7 +83,7 @@ int validate(const void *q, const void *k, const void *v, const void *o, const v
     if (H % Hkv != 0) return AVE_ERR_BAD_SHAPE;
     if (Sq >= (1 << 30) || Sk >= (1 << 30)) return AVE_ERR_BAD_SHAPE;
     if ((long long)B * H >= (1ll << 31)) return AVE_ERR_BAD_SHAPE;
-    if (D != 64 && D != 128) return AVE_ERR_UNSUPPORTED_D;
+    if (D < 8 || D > 128 || D % 8 != 0) return AVE_ERR_UNSUPPORTED_D;
     const long long n_qblk = (Sq + ave::BM - 1) / ave::BM;
     if (n_qblk * B * H >= (1ll << 31)) return AVE_ERR_BAD_SHAPE;
     return -1;  // shape checks passed; pointer/scale checks follow
@@ -165,6 +165,11 @@ int launch_attention(const void *q, const void *k, const void *v, void *o, float
     ave::FwdParams p;
     p.o = o;
     p.lse = lse;
+    p.o_stride_b = so.batch;
+    p.o_stride_h = so.head;
+    p.o_stride_r = so.row;
+    p.d_true = D;
+    const int Dk = D <= 64 ? 64 : 128;  // the kernel's head dimension: TMA zero-fills the columns beyond D
     p.H = H;
     p.Hkv = Hkv;
     p.Sq = Sq;
@@ -195,11 +200,11 @@ int launch_attention(const void *q, const void *k, const void *v, void *o, float
     p.scale_log2 = scale * 1.4426950408889634f;
 
     if (split) {
-        if (D == 128)
+        if (Dk == 128)
             return causal ? launch_ws<128, true, true>(tq, tk, tv, to, p, s) : launch_ws<128, false, true>(tq, tk, tv, to, p, s);
         return causal ? launch_ws<64, true, true>(tq, tk, tv, to, p, s) : launch_ws<64, false, true>(tq, tk, tv, to, p, s);
     }
-    if (D == 128)
+    if (Dk == 128)
         return causal ? launch_ws<128, true, false>(tq, tk, tv, to, p, s) : launch_ws<128, false, false>(tq, tk, tv, to, p, s);
     return causal ? launch_ws<64, true, false>(tq, tk, tv, to, p, s) : launch_ws<64, false, false>(tq, tk, tv, to, p, s);
 }
@@ -374,6 +379,7 @@ int ave_attn_fwd_splitkv(const void *q, const void *k, const void *v, void *o, f
                          size_t workspace_bytes, void *stream) {
     int st = validate(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, scale);
     if (st >= 0) return st;
+    if (D != 64 && D != 128) return AVE_ERR_UNSUPPORTED_D;
     if (n_splits < 1 || n_splits > AVE_SPLITKV_MAX_SPLITS) return AVE_ERR_BAD_SHAPE;
     st = validate_ptrs_and_scale(q, k, v, o, lse, scale);
     if (st != AVE_OK) return st;
@@ -394,6 +400,7 @@ int ave_attn_fwd_splitkv_static(const void *q, const void *k, const void *v, voi
                                 void *stream) {
     int st = validate(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, scale);
     if (st >= 0) return st;
+    if (D != 64 && D != 128) return AVE_ERR_UNSUPPORTED_D;
     if (n_splits < 1 || n_splits > AVE_SPLITKV_MAX_SPLITS) return AVE_ERR_BAD_SHAPE;
     st = validate_ptrs_and_scale(q, k, v, o, lse, scale);
     if (st != AVE_OK) return st;
@@ -451,7 +458,7 @@ const char *ave_attn_strerror(int status) {
         case AVE_OK: return "ok";
         case AVE_ERR_NULL_POINTER: return "a required pointer is NULL";
         case AVE_ERR_BAD_SHAPE: return "bad shape: sizes must be positive, H a multiple of Hkv, and within limits";
-        case AVE_ERR_UNSUPPORTED_D: return "unsupported head dimension (D must be 64 or 128)";
+        case AVE_ERR_UNSUPPORTED_D: return "unsupported head dimension (a multiple of 8 up to 128; 64 or 128 for the split-KV calls)";
         case AVE_ERR_MISALIGNED: return "q, k, v, o must be 16-byte aligned and lse 4-byte aligned";
         case AVE_ERR_BAD_SCALE: return "scale is NaN or infinite";
         case AVE_ERR_UNSUPPORTED_DEVICE: return "the current CUDA device is not compute capability 10.x";

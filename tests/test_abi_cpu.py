@@ -58,7 +58,7 @@ def test_validation_order_before_any_cuda_call(lib):
     assert f(A, A, A, A, A, 1, 2, 2, -5, 128, 64, 0, 1.0) == binding.AVE_ERR_BAD_SHAPE
     assert f(A, A, A, A, A, 1, 6, 4, 128, 128, 64, 0, 1.0) == binding.AVE_ERR_BAD_SHAPE      # H % Hkv
     assert f(A, A, A, A, A, 1, 2, 2, 1 << 30, 128, 64, 0, 1.0) == binding.AVE_ERR_BAD_SHAPE
-    assert f(A, A, A, A, A, 1, 2, 2, 128, 128, 96, 0, 1.0) == binding.AVE_ERR_UNSUPPORTED_D
+    assert f(A, A, A, A, A, 1, 2, 2, 128, 128, 100, 0, 1.0) == binding.AVE_ERR_UNSUPPORTED_D
     assert f(A, A, A, A, A, 1, 2, 2, 128, 128, 256, 0, 1.0) == binding.AVE_ERR_UNSUPPORTED_D
     assert f(A + 8, A, A, A, A, 1, 2, 2, 128, 128, 64, 0, 1.0) == binding.AVE_ERR_MISALIGNED
     assert f(A, A, A, A + 2, A, 1, 2, 2, 128, 128, 64, 0, 1.0) == binding.AVE_ERR_MISALIGNED
@@ -66,7 +66,7 @@ def test_validation_order_before_any_cuda_call(lib):
     assert f(A, A, A, A, A, 1, 2, 2, 128, 128, 64, 0, float("inf")) == binding.AVE_ERR_BAD_SCALE
     assert f(A, A, A, A, A, 1, 2, 2, 128, 128, 64, 0, float("nan")) == binding.AVE_ERR_BAD_SCALE
     # bad D outranks misalignment, bad shape outranks bad D (order of the status codes)
-    assert f(A + 8, A, A, A, A, 1, 2, 2, 128, 128, 96, 0, 1.0) == binding.AVE_ERR_UNSUPPORTED_D
+    assert f(A + 8, A, A, A, A, 1, 2, 2, 128, 128, 100, 0, 1.0) == binding.AVE_ERR_UNSUPPORTED_D
     assert f(A, A, A, A, A, 1, 3, 2, 128, 128, 96, 0, 1.0) == binding.AVE_ERR_BAD_SHAPE
 
 
@@ -85,7 +85,7 @@ def test_host_workspace_bytes(lib):
     q = 4 * 32 * 2048 * 128 * 2
     assert n == 4 * q + 4 * 32 * 2048 * 4
     assert binding.host_workspace_bytes(1, 3, 2, 8, 8, 64) == 0      # invalid shape
-    assert binding.host_workspace_bytes(1, 2, 2, 8, 8, 32) == 0      # unsupported D
+    assert binding.host_workspace_bytes(1, 2, 2, 8, 8, 36) == 0      # unsupported D
     assert binding.host_workspace_bytes(1, 1, 1, 1, 1, 64) == 256 * 5  # each buffer rounded up to 256 B
 
 

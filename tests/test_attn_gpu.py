@@ -81,6 +81,34 @@ def test_seeded_random_shapes(B, H, Hkv, Sq, Sk, D, causal, scale):
     parity.check_full(q, k, v, causal, scale, "random shape %s" % ((B, H, Hkv, Sq, Sk, D, causal, scale),))
 
 
+@pytest.mark.parametrize("D", [8, 32, 40, 72, 96, 120])
+@pytest.mark.parametrize("causal", [False, True])
+def test_head_dimensions_other_than_64_and_128(D, causal):
+    """D is any multiple of 8 up to 128: the loads zero-fill and the stores clip the columns beyond D."""
+    q, k, v = rand_qkv(900 + D, 2, 4, 2, 200, 333, D)
+    parity.check_full(q, k, v, causal, 1.0 / math.sqrt(D), "D = %d" % D)
+
+
+def test_rows_without_keys_in_a_strided_output():
+    """Causal with Sq > Sk: the leading rows see no key and are written as zeros through O's strides."""
+    B, H, Sq, Sk, D = 2, 3, 400, 130, 96
+    q, k, v = rand_qkv(77, B, H, H, Sq, Sk, D)
+    scale = 1.0 / math.sqrt(D)
+    dev = "cuda:0"
+    qs, ks, vs = (t.permute(0, 2, 1, 3).contiguous().to(dev) for t in (q, k, v))   # (B, S, H, D) storage
+    os_ = torch.full((B, Sq, H, D + 8), 777.0, dtype=torch.bfloat16, device=dev)      # padded rows
+    ov = os_[..., :D].permute(0, 2, 1, 3)
+    ov.fill_(float("nan"))
+    o, lse = binding.ave_attn_fwd_strided(qs.permute(0, 2, 1, 3), ks.permute(0, 2, 1, 3), vs.permute(0, 2, 1, 3), ov,
+                                          causal=True, scale=scale)
+    st, raw = binding.device_status()
+    assert st == binding.AVE_OK, "device status %d raw %#x" % (st, raw)
+    o_ref, lse_ref = oracle.attn_fwd(q, k, v, True, scale)
+    parity.compare(ov.cpu().contiguous(), lse.cpu(), o_ref, lse_ref, "strided, rows without keys")
+    assert torch.all(os_[..., D:] == 777.0), "padding between O rows was written"
+    assert torch.all(ov[:, :, :Sq - Sk] == 0) and torch.all(torch.isinf(lse[:, :, :Sq - Sk]))
+
+
 @pytest.mark.parametrize("scale", [0.0, -0.1, 0.02, 0.3])
 @pytest.mark.parametrize("causal", [False, True])
 def test_scale_values_including_zero_and_negative(scale, causal):
@@ -165,7 +193,7 @@ def test_errors_launch_nothing_and_leave_outputs_alone():
     lse = torch.full((1, 2, 128), 5.0, device=dev)
     n0 = binding.launch_count()
     P = lambda t: t.data_ptr()
-    assert binding.ave_attn_fwd_raw(P(q), P(q), P(q), P(o), P(lse), 1, 2, 2, 128, 128, 96, 0, 1.0) == binding.AVE_ERR_UNSUPPORTED_D
+    assert binding.ave_attn_fwd_raw(P(q), P(q), P(q), P(o), P(lse), 1, 2, 2, 128, 128, 100, 0, 1.0) == binding.AVE_ERR_UNSUPPORTED_D
     assert binding.ave_attn_fwd_raw(P(q) + 2, P(q), P(q), P(o), P(lse), 1, 2, 2, 128, 128, 64, 0, 1.0) == binding.AVE_ERR_MISALIGNED
     assert binding.ave_attn_fwd_raw(P(q), P(q), P(q), P(o), P(lse), 1, 3, 2, 128, 128, 64, 0, 1.0) == binding.AVE_ERR_BAD_SHAPE
     assert binding.ave_attn_fwd_raw(P(q), P(q), P(q), P(o), P(lse), 1, 2, 2, 128, 128, 64, 0, float("nan")) == binding.AVE_ERR_BAD_SCALE
