@@ -93,6 +93,30 @@ int ave_attn_fwd_strided(const void *q, const void *k, const void *v, void *o, f
                          int causal, float scale, void *stream);
 
 /*
+ * The same operation for a batch of sequences of different lengths packed
+ * without padding ("varlen").  Token-major DEVICE tensors:
+ *   q   bf16 [total_q, H,   D]   read       k, v  bf16 [total_k, Hkv, D]   read
+ *   o   bf16 [total_q, H,   D]   written    lse   fp32 [H, total_q]        written
+ * Sequence b (0 <= b < B) owns query rows [cu_seqlens_q[b], cu_seqlens_q[b+1])
+ * and key rows [cu_seqlens_k[b], cu_seqlens_k[b+1]); attention is computed
+ * inside each sequence only, with that sequence's own lengths in the causal
+ * rule j <= i + (Sk_b - Sq_b).  cu_seqlens_q and cu_seqlens_k are DEVICE arrays
+ * of B + 1 non-decreasing int32 values starting at 0 and ending at total_q and
+ * total_k; they are read by the kernel, not by the host, so they are not
+ * validated: a sequence longer than max_Sq (queries) or max_Sk (keys), or
+ * offsets outside [0, total], give undefined results.  Sequences of length 0
+ * are allowed; a sequence with queries but no keys gets O = 0, LSE = -inf.
+ * max_Sq / max_Sk: upper bounds of the sequences' lengths (they size the launch;
+ * tighter is faster), 1 <= max_Sq <= total_q, 1 <= max_Sk <= total_k.
+ * D, H, Hkv, causal, scale, stream, validation order and error behaviour as for
+ * ave_attn_fwd.
+ */
+int ave_attn_fwd_varlen(const void *q, const void *k, const void *v, void *o, float *lse,
+                        const int *cu_seqlens_q, const int *cu_seqlens_k,
+                        int B, int H, int Hkv, int max_Sq, int max_Sk, int total_q, int total_k,
+                        int D, int causal, float scale, void *stream);
+
+/*
  * The same operation for tensors that live in HOST memory (same layouts and
  * limits).  The call enqueues, on `stream`: host-to-device copies of q, k, v
  * into `workspace`, the attention kernel, and device-to-host copies of o and

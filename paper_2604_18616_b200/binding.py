@@ -51,6 +51,8 @@ def lib() -> ctypes.CDLL:
         L.ave_attn_fwd.restype = ci
         L.ave_attn_fwd_strided.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, vp, vp, vp, vp, ci, cf, vp]
         L.ave_attn_fwd_strided.restype = ci
+        L.ave_attn_fwd_varlen.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp]
+        L.ave_attn_fwd_varlen.restype = ci
         L.ave_attn_fwd_host.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, cf, vp, ctypes.c_size_t, vp]
         L.ave_attn_fwd_host.restype = ci
         L.ave_attn_host_workspace_bytes.argtypes = [ci] * 6
@@ -167,6 +169,39 @@ def ave_attn_fwd_strided(q, k, v, o, lse=None, causal=False, scale=None, stream=
             int(bool(causal)), float(scale), _stream_ptr(stream))
     if st != AVE_OK:
         raise AveAttnError(st, "ave_attn_fwd_strided")
+    return o, lse
+
+
+def ave_attn_fwd_varlen(q, k, v, cu_seqlens_q, cu_seqlens_k, max_sq, max_sk, o=None, lse=None, causal=False,
+                        scale=None, stream=None):
+    """Variable-length batch: q [total_q,H,D], k/v [total_k,Hkv,D] contiguous CUDA bf16, cu_seqlens_* CUDA int32
+    [B+1].  Returns o [total_q,H,D] bf16 and lse [H,total_q] fp32."""
+    for t in (q, k, v):
+        if not (t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous() and t.dim() == 3):
+            raise ValueError("q, k, v must be contiguous 3-D CUDA bfloat16 tensors")
+    for t in (cu_seqlens_q, cu_seqlens_k):
+        if not (t.is_cuda and t.dtype == torch.int32 and t.is_contiguous() and t.dim() == 1):
+            raise ValueError("cu_seqlens must be contiguous 1-D CUDA int32 tensors")
+    total_q, H, D = q.shape
+    total_k, Hkv, Dk = k.shape
+    B = cu_seqlens_q.numel() - 1
+    if tuple(v.shape) != tuple(k.shape) or Dk != D or cu_seqlens_k.numel() != B + 1:
+        raise ValueError("inconsistent shapes")
+    if o is None:
+        o = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((H, total_q), dtype=torch.float32, device=q.device)
+    if scale is None:
+        scale = D ** -0.5
+    with torch.cuda.device(q.device):
+        st = lib().ave_attn_fwd_varlen(
+            ctypes.c_void_p(q.data_ptr()), ctypes.c_void_p(k.data_ptr()), ctypes.c_void_p(v.data_ptr()),
+            ctypes.c_void_p(o.data_ptr()), ctypes.c_void_p(lse.data_ptr()),
+            ctypes.c_void_p(cu_seqlens_q.data_ptr()), ctypes.c_void_p(cu_seqlens_k.data_ptr()),
+            B, H, Hkv, int(max_sq), int(max_sk), total_q, total_k, D, int(bool(causal)), float(scale),
+            _stream_ptr(stream))
+    if st != AVE_OK:
+        raise AveAttnError(st, "ave_attn_fwd_varlen")
     return o, lse
 
 

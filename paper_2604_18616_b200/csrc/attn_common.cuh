@@ -46,6 +46,10 @@ struct FwdParams {
     int n_splits;
     int keys_per_split;
     int rows_per_head;   // > 0: rows are (query head in group, query position) pairs, this many positions per head
+    // Variable-length launches only: sequence b owns query rows [cu_q[b], cu_q[b+1]) and key rows
+    // [cu_k[b], cu_k[b+1]) of token-major tensors [rows, heads, D]; Sq and Sk above are the maxima.
+    const int *cu_q, *cu_k;        // device, B + 1 entries each
+    long long lse_stride_h;        // lse is [H, total query rows]
     float *o_partial;    // fp32 [n_splits, B*H, Sq, D]
     float *lse_partial;  // fp32 [n_splits, B*H, Sq]
 };

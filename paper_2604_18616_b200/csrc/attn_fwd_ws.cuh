@@ -96,6 +96,14 @@ struct WorkTileT<true> : WorkTileBase {
     int split;           // index of the key range
 };
 
+// Variable-length launches (never split): the tile also carries its sequence's lengths and first rows.
+struct WorkTileVar : WorkTileT<false> {
+    int sq, sk;          // this sequence's query and key counts
+    int q_base, k_base;  // its first row in the token-major Q/O and K/V tensors
+};
+template <bool SPLIT, bool VARLEN>
+using TileOf = std::conditional_t<VARLEN, WorkTileVar, WorkTileT<SPLIT>>;
+
 // Split-KV launches may pack the G query heads of a key/value head into the rows of one problem
 // ("head" = KV head, row r = head_in_group * rows_per_head + query position): the rows of Q, O and LSE
 // are contiguous that way, and only the causal mask needs the query position r % rows_per_head.
@@ -136,9 +144,10 @@ __device__ __forceinline__ int kv_tiles_whole(int i0, int Sq, int Sk) {
 // fit in L2 together); inside a group all heads' blocks of one query position,
 // longest (causal: last) position first.  Split-KV: the key ranges of one
 // (b, h, block) are adjacent in the order.
-template <bool CAUSAL, bool SPLIT>
-__device__ __forceinline__ WorkTileT<SPLIT> decode_tile(int id, const FwdParams &p) {
-    WorkTileT<SPLIT> w;
+template <bool CAUSAL, bool SPLIT, bool VARLEN = false>
+__device__ __forceinline__ TileOf<SPLIT, VARLEN> decode_tile(int id, const FwdParams &p) {
+    static_assert(!(SPLIT && VARLEN), "variable-length launches are not split");
+    TileOf<SPLIT, VARLEN> w;
     int k_begin = 0, k_end = p.Sk;
     if constexpr (SPLIT) {
         w.split = id % p.n_splits;
@@ -161,6 +170,15 @@ __device__ __forceinline__ WorkTileT<SPLIT> decode_tile(int id, const FwdParams 
     if constexpr (SPLIT) {
         w.n0 = kv_tiles_for<CAUSAL>(query_pos_hi(w.q0, p.rows_per_head), p.causal_off, k_begin, k_end);
         w.n1 = max(w.n0, kv_tiles_for<CAUSAL>(query_pos_hi(w.q0 + BM, p.rows_per_head), p.causal_off, k_begin, k_end));
+    } else if constexpr (VARLEN) {
+        w.q_base = p.cu_q[w.b];
+        w.k_base = p.cu_k[w.b];
+        w.sq = p.cu_q[w.b + 1] - w.q_base;
+        w.sk = p.cu_k[w.b + 1] - w.k_base;
+        // sub-tiles that start beyond the sequence's last query row have no rows and visit no keys
+        w.n0 = (w.q0 < w.sq && w.sk > 0) ? kv_tiles_whole<CAUSAL>(w.q0, w.sq, w.sk) : 0;
+        w.n1 = (w.q0 + BM < w.sq && w.sk > 0) ? kv_tiles_whole<CAUSAL>(w.q0 + BM, w.sq, w.sk) : 0;
+        w.n1 = max(w.n0, w.n1);
     } else {
         w.n0 = kv_tiles_whole<CAUSAL>(w.q0, p.Sq, p.Sk);
         w.n1 = kv_tiles_whole<CAUSAL>(w.q0 + BM, p.Sq, p.Sk);
@@ -174,6 +192,26 @@ __device__ __forceinline__ int key_end(const WorkTileT<false> &, const FwdParams
 __device__ __forceinline__ int key_end(const WorkTileT<true> &w, const FwdParams &) { return w.k_end; }
 __device__ __forceinline__ int split_of(const WorkTileT<false> &) { return 0; }
 __device__ __forceinline__ int split_of(const WorkTileT<true> &w) { return w.split; }
+__device__ __forceinline__ int key_end(const WorkTileVar &w, const FwdParams &) { return w.sk; }
+// Query/key counts and first rows of the tile's sequence; the tensor-map batch coordinate.
+template <class Tile> __device__ __forceinline__ int seq_q(const Tile &, const FwdParams &p) { return p.Sq; }
+template <class Tile> __device__ __forceinline__ int seq_k(const Tile &, const FwdParams &p) { return p.Sk; }
+template <class Tile> __device__ __forceinline__ int q_base_of(const Tile &) { return 0; }
+template <class Tile> __device__ __forceinline__ int k_base_of(const Tile &) { return 0; }
+template <class Tile> __device__ __forceinline__ int batch_coord(const Tile &w) { return w.b; }
+__device__ __forceinline__ int seq_q(const WorkTileVar &w, const FwdParams &) { return w.sq; }
+__device__ __forceinline__ int seq_k(const WorkTileVar &w, const FwdParams &) { return w.sk; }
+__device__ __forceinline__ int q_base_of(const WorkTileVar &w) { return w.q_base; }
+__device__ __forceinline__ int k_base_of(const WorkTileVar &w) { return w.k_base; }
+__device__ __forceinline__ int batch_coord(const WorkTileVar &) { return 0; }
+// Index of row i's log-sum-exp: [B, H, Sq], or [H, total rows] for variable-length launches.
+template <class Tile>
+__device__ __forceinline__ size_t lse_index(const Tile &w, const FwdParams &p, int i) {
+    return size_t(w.bh) * p.Sq + i;
+}
+__device__ __forceinline__ size_t lse_index(const WorkTileVar &w, const FwdParams &p, int i) {
+    return size_t(w.h) * p.lse_stride_h + w.q_base + i;
+}
 
 // ---- cluster launch control: take over the tile of a CTA that has not started
 __device__ __forceinline__ void clc_try_cancel(uint32_t response_smem, uint32_t bar) {
@@ -199,7 +237,7 @@ __device__ __forceinline__ int clc_decode(const volatile unsigned long long *res
     return ok ? int(x) : -1;
 }
 
-template <int D, bool CAUSAL, bool SPLIT>
+template <int D, bool CAUSAL, bool SPLIT, bool VARLEN = false>
 __global__ void __launch_bounds__(384, 1)
 attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
@@ -311,7 +349,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             bool ok = true;
             int id = blockIdx.x;
             for (int n = 0; id >= 0 && ok; ++n) {
-                const WorkTileT<SPLIT> w = decode_tile<CAUSAL, SPLIT>(id, p);
+                const TileOf<SPLIT, VARLEN> w = decode_tile<CAUSAL, SPLIT, VARLEN>(id, p);
                 // Q_t of this tile goes in as soon as the previous tile's last Q_t K^T has retired.
                 // Q_1 is released later than Q_0 (causal sub-tile 1 runs one step longer), and the
                 // first K/V tiles must not queue behind it, so a Q load that cannot go yet stays
@@ -333,7 +371,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         mbar_arrive_expect_tx(bar, Cfg::kTileBytes);
                         for (int x = 0; x < Cfg::kBoxes; ++x)  // the tensor maps are {D, rows, heads, batch}
                             tma_load_4d(sQ + t * Cfg::kTileBytes + x * Cfg::kBoxBytes, &tm_q, bar, x * 64,
-                                        w.q0 + t * BM, w.h, w.b);
+                                        q_base_of(w) + w.q0 + t * BM, w.h, batch_coord(w));
                     }
                 };
                 try_load_q(0, false);
@@ -372,7 +410,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         mbar_arrive_expect_tx(bar, Cfg::kTileBytes);
                         for (int x = 0; x < Cfg::kBoxes; ++x)
                             tma_load_4d(sRing + slot * Cfg::kTileBytes + x * Cfg::kBoxBytes, tm, bar, x * 64,
-                                        key_begin(w) + (it >> 1) * BN, w.g, w.b);
+                                        k_base_of(w) + key_begin(w) + (it >> 1) * BN, w.g, batch_coord(w));
                     }
                 }
                 if (ok) try_load_q(0, true);
@@ -430,7 +468,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             // First step of sub-tile t in tile number `tn` (tile `wt`, whose K_0 sits at ring position
             // `ring0`): S_t = Q_t K_0^T.  Issued as soon as sub-tile t has finished the tile before, so
             // the next tile's first scores are computed while the other sub-tile is still at work.
-            auto start_subtile = [&](int t, const WorkTileT<SPLIT> &wt, int tn, int ring0) {
+            auto start_subtile = [&](int t, const TileOf<SPLIT, VARLEN> &wt, int tn, int ring0) {
                 const int n_t = t ? wt.n1 : wt.n0;
                 ok = wait_bar(&bar_q_full[t], tn & 1, STATUS_TIMEOUT_LOAD);
                 if (ok && n_t > 0) ok = wait_full(ring0);
@@ -446,7 +484,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             };
 
             int id = blockIdx.x;
-            WorkTileT<SPLIT> w = decode_tile<CAUSAL, SPLIT>(id, p);
+            TileOf<SPLIT, VARLEN> w = decode_tile<CAUSAL, SPLIT, VARLEN>(id, p);
             start_subtile(0, w, 0, 0);
             if (ok) start_subtile(1, w, 0, 0);
             for (int n = 0; id >= 0 && ok; ++n) {
@@ -455,8 +493,8 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 // the tile after this one (its first steps are issued from inside this tile's loop)
                 const int id_next = next_tile(n, ok);
                 if (!ok) break;
-                WorkTileT<SPLIT> w_next = w;
-                if (id_next >= 0) w_next = decode_tile<CAUSAL, SPLIT>(id_next, p);
+                TileOf<SPLIT, VARLEN> w_next = w;
+                if (id_next >= 0) w_next = decode_tile<CAUSAL, SPLIT, VARLEN>(id_next, p);
                 const int ring_next = ring + 2 * n1;
                 if (id_next >= 0 && n1 == 0) {  // nothing to do in this tile at all
                     start_subtile(0, w_next, n + 1, ring_next);
@@ -527,7 +565,6 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const int t = (warp - 4) >> 2;                // sub-tile
         const int wq = warp & 3;                      // TMEM lane quadrant of this warp
         const int r = wq * 32 + lane;                 // row within the sub-tile = TMEM lane
-        const int off = SPLIT ? p.causal_off : p.Sk - p.Sq;
         const uint32_t lane_sel = uint32_t(wq * 32) << 16;
         const uint32_t tS = tmem + (t ? Cfg::kColS1 : Cfg::kColS0) + lane_sel;
         const uint32_t tO = tmem + (t ? Cfg::kColO1 : Cfg::kColO0) + lane_sel;
@@ -542,25 +579,27 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 
         int id = blockIdx.x;
         for (int n = 0; id >= 0 && ok; ++n) {
-            const WorkTileT<SPLIT> w = decode_tile<CAUSAL, SPLIT>(id, p);
+            const TileOf<SPLIT, VARLEN> w = decode_tile<CAUSAL, SPLIT, VARLEN>(id, p);
             const int bh = w.bh;
+            const int sq = seq_q(w, p);                // query rows of this tile's sequence
+            const int off = SPLIT ? p.causal_off : seq_k(w, p) - sq;
             const int i0 = w.q0 + t * BM;
             const int i = i0 + r;                     // query row
             const int n_t = t ? w.n1 : w.n0;
 
             if (n_t == 0) {
                 // no key visible to any row of this sub-tile: O = 0, LSE = -inf
-                if (i < p.Sq) {
+                if (i < sq) {
                     const uint4 z = make_uint4(0, 0, 0, 0);
                     if (SPLIT) {
                         const size_t row = (size_t(split_of(w)) * p.BH + bh) * p.Sq + i;
                         for (int c = 0; c < D / 4; ++c) reinterpret_cast<uint4 *>(p.o_partial + row * D)[c] = z;
                         p.lse_partial[row] = -INFINITY;
                     } else {
-                        __nv_bfloat16 *o_row = reinterpret_cast<__nv_bfloat16 *>(p.o) + w.b * p.o_stride_b +
-                                               w.h * p.o_stride_h + i * p.o_stride_r;
+                        __nv_bfloat16 *o_row = reinterpret_cast<__nv_bfloat16 *>(p.o) + batch_coord(w) * p.o_stride_b +
+                                               w.h * p.o_stride_h + (q_base_of(w) + i) * p.o_stride_r;
                         for (int c = 0; c < p.d_true / 8; ++c) reinterpret_cast<uint4 *>(o_row)[c] = z;
-                        p.lse[size_t(bh) * p.Sq + i] = -INFINITY;
+                        p.lse[lse_index(w, p, i)] = -INFINITY;
                     }
                 }
                 // O_t was not used: hand it back at once so its barrier completes once per tile
@@ -768,7 +807,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&bar_o_free[t]));
                     } else {
-                    if (i < p.Sq) p.lse[size_t(bh) * p.Sq + i] = lse_row;
+                    if (i < sq) p.lse[lse_index(w, p, i)] = lse_row;
 #pragma unroll
                     for (int x = 0; x < Cfg::kBoxes; ++x) {  // 64 columns of O at a time through the staging rows
                         uint32_t oc[2][32];
@@ -780,6 +819,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                             __syncwarp();
                             if (lane == 0) mbar_arrive(smem_u32(&bar_o_free[t]));
                         }
+                        // Variable-length launches: a 32-row box that reaches past the sequence's last row would
+                        // overwrite the next sequence's rows, so that warp stores its rows one by one instead.
+                        const bool whole_box = !VARLEN || (i0 + wq * 32 + 32 <= sq);
                         // this warp's previous TMA store must have finished reading the staging rows
                         if (lane == 0 && store_pending) tma_store_wait_read();
                         __syncwarp();
@@ -793,14 +835,20 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                             v4.w = pack_bf16x2(__uint_as_float(src[6]) * inv_l, __uint_as_float(src[7]) * inv_l);
                             // 16-byte chunk `ch` of row `lane`, in the 128-byte-swizzled layout TMA expects
                             const int ch = e >> 3;
-                            const uint32_t addr = sO + lane * 128 + ((ch ^ (lane & 7)) << 4);
-                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v4.x), "r"(v4.y),
-                                         "r"(v4.z), "r"(v4.w) : "memory");
+                            if (whole_box) {
+                                const uint32_t addr = sO + lane * 128 + ((ch ^ (lane & 7)) << 4);
+                                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v4.x), "r"(v4.y),
+                                             "r"(v4.z), "r"(v4.w) : "memory");
+                            } else if (i < sq && x * 64 + e < p.d_true) {
+                                __nv_bfloat16 *o_row = reinterpret_cast<__nv_bfloat16 *>(p.o) + w.h * p.o_stride_h +
+                                                       (q_base_of(w) + i) * p.o_stride_r;
+                                *reinterpret_cast<uint4 *>(o_row + x * 64 + e) = v4;
+                            }
                         }
                         fence_proxy_async_smem();
                         __syncwarp();
-                        if (lane == 0 && i0 + wq * 32 < p.Sq) {
-                            tma_store_4d(&tm_o, sO, x * 64, i0 + wq * 32, w.h, w.b);
+                        if (lane == 0 && whole_box && i0 + wq * 32 < sq) {
+                            tma_store_4d(&tm_o, sO, x * 64, q_base_of(w) + i0 + wq * 32, w.h, batch_coord(w));
                             tma_store_commit();
                             store_pending = true;
                         }

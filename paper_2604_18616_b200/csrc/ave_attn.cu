@@ -119,11 +119,11 @@ int check_device() {
     return AVE_OK;
 }
 
-template <int D, bool CAUSAL, bool SPLIT>
+template <int D, bool CAUSAL, bool SPLIT, bool VARLEN = false>
 int launch_ws(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const CUtensorMap &to,
               const ave::FwdParams &p, cudaStream_t stream) {
     using Cfg = ave::WsCfg<D>;
-    auto kern = ave::attn_fwd_ws_kernel<D, CAUSAL, SPLIT>;
+    auto kern = ave::attn_fwd_ws_kernel<D, CAUSAL, SPLIT, VARLEN>;
     static std::atomic<bool> configured{false};  // per instantiation
     if (!configured.load(std::memory_order_acquire)) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
@@ -147,19 +147,29 @@ int launch_ws(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &t
 // Encode the tensor maps, fill the kernel parameters and launch.  n_splits == 1 with no partial
 // buffers is the ordinary forward; otherwise every work tile covers one range of keys_per_split keys
 // and writes fp32 partials.
-// `layout` (strides of q, k, v, o in this order) is NULL for contiguous [B, heads, rows, D] tensors.
+// Variable-length launch: token-major tensors [rows, heads, D] and the sequences' row ranges.
+struct VarlenArgs {
+    const int *cu_q, *cu_k;  // device, B + 1 entries
+    int total_q, total_k;
+};
+
+// `layout` (strides of q, k, v, o in this order) is NULL for contiguous [B, heads, rows, D] tensors; `varlen`
+// is NULL unless the launch is a variable-length one (Sq and Sk are then the longest sequences).
 int launch_attention(const void *q, const void *k, const void *v, void *o, float *lse, int B, int H, int Hkv, int Sq,
                      int Sk, int D, int causal, float scale, int n_splits, int keys_per_split, float *o_partial,
-                     float *lse_partial, int rows_per_head, const Strides *layout, cudaStream_t s) {
-    const Strides sq = layout ? layout[0] : contiguous_strides(H, Sq, D);
-    const Strides sk = layout ? layout[1] : contiguous_strides(Hkv, Sk, D);
-    const Strides sv = layout ? layout[2] : contiguous_strides(Hkv, Sk, D);
-    const Strides so = layout ? layout[3] : contiguous_strides(H, Sq, D);
+                     float *lse_partial, int rows_per_head, const Strides *layout, const VarlenArgs *varlen,
+                     cudaStream_t s) {
+    auto token_major = [&](int heads, int rows) { return Strides{(long long)rows * heads * D, (long long)D, (long long)heads * D}; };
+    const int rows_q = varlen ? varlen->total_q : Sq, rows_k = varlen ? varlen->total_k : Sk, n_batch = varlen ? 1 : B;
+    const Strides sq = layout ? layout[0] : varlen ? token_major(H, rows_q) : contiguous_strides(H, Sq, D);
+    const Strides sk = layout ? layout[1] : varlen ? token_major(Hkv, rows_k) : contiguous_strides(Hkv, Sk, D);
+    const Strides sv = layout ? layout[2] : varlen ? token_major(Hkv, rows_k) : contiguous_strides(Hkv, Sk, D);
+    const Strides so = layout ? layout[3] : varlen ? token_major(H, rows_q) : contiguous_strides(H, Sq, D);
     CUtensorMap tq, tk, tv, to;
-    if (!encode_map(&tq, q, D, Sq, H, B, sq, ave::BM)) return AVE_ERR_CUDA;
-    if (!encode_map(&to, o, D, Sq, H, B, so, ave::WsCfg<128>::kOutBoxRows)) return AVE_ERR_CUDA;
-    if (!encode_map(&tk, k, D, Sk, Hkv, B, sk, ave::BN)) return AVE_ERR_CUDA;
-    if (!encode_map(&tv, v, D, Sk, Hkv, B, sv, ave::BN)) return AVE_ERR_CUDA;
+    if (!encode_map(&tq, q, D, rows_q, H, n_batch, sq, ave::BM)) return AVE_ERR_CUDA;
+    if (!encode_map(&to, o, D, rows_q, H, n_batch, so, ave::WsCfg<128>::kOutBoxRows)) return AVE_ERR_CUDA;
+    if (!encode_map(&tk, k, D, rows_k, Hkv, n_batch, sk, ave::BN)) return AVE_ERR_CUDA;
+    if (!encode_map(&tv, v, D, rows_k, Hkv, n_batch, sv, ave::BN)) return AVE_ERR_CUDA;
 
     const bool split = o_partial != nullptr;
     ave::FwdParams p;
@@ -169,6 +179,9 @@ int launch_attention(const void *q, const void *k, const void *v, void *o, float
     p.o_stride_h = so.head;
     p.o_stride_r = so.row;
     p.d_true = D;
+    p.cu_q = varlen ? varlen->cu_q : nullptr;
+    p.cu_k = varlen ? varlen->cu_k : nullptr;
+    p.lse_stride_h = varlen ? varlen->total_q : 0;
     const int Dk = D <= 64 ? 64 : 128;  // the kernel's head dimension: TMA zero-fills the columns beyond D
     p.H = H;
     p.Hkv = Hkv;
@@ -203,6 +216,13 @@ int launch_attention(const void *q, const void *k, const void *v, void *o, float
         if (Dk == 128)
             return causal ? launch_ws<128, true, true>(tq, tk, tv, to, p, s) : launch_ws<128, false, true>(tq, tk, tv, to, p, s);
         return causal ? launch_ws<64, true, true>(tq, tk, tv, to, p, s) : launch_ws<64, false, true>(tq, tk, tv, to, p, s);
+    }
+    if (varlen) {
+        if (Dk == 128)
+            return causal ? launch_ws<128, true, false, true>(tq, tk, tv, to, p, s)
+                          : launch_ws<128, false, false, true>(tq, tk, tv, to, p, s);
+        return causal ? launch_ws<64, true, false, true>(tq, tk, tv, to, p, s)
+                      : launch_ws<64, false, false, true>(tq, tk, tv, to, p, s);
     }
     if (Dk == 128)
         return causal ? launch_ws<128, true, false>(tq, tk, tv, to, p, s) : launch_ws<128, false, false>(tq, tk, tv, to, p, s);
@@ -260,9 +280,9 @@ int run_splitkv(const void *q, const void *k, const void *v, void *o, float *lse
     const int G = H / Hkv;
     const bool pack = G > 1 && Sq < 2 * ave::BM && (long long)G * Sq < (1ll << 30);
     int st = pack ? launch_attention(q, k, v, o, lse, B, Hkv, Hkv, G * Sq, Sk, D, causal, scale, n_splits, kps,
-                                     o_partial, lse_partial, Sq, nullptr, s)
+                                     o_partial, lse_partial, Sq, nullptr, nullptr, s)
                   : launch_attention(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, causal, scale, n_splits, kps, o_partial,
-                                     lse_partial, 0, nullptr, s);
+                                     lse_partial, 0, nullptr, nullptr, s);
     if (st != AVE_OK) return st;
     const long long rows = (long long)B * H * Sq;
     const long long work = rows * (D / 8);
@@ -291,7 +311,7 @@ int ave_attn_fwd(const void *q, const void *k, const void *v, void *o, float *ls
     st = check_device();
     if (st != AVE_OK) return st;
     return launch_attention(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, causal, scale, 1, 0, nullptr, nullptr, 0, nullptr,
-                            static_cast<cudaStream_t>(stream));
+                            nullptr, static_cast<cudaStream_t>(stream));
 }
 
 int ave_attn_fwd_strided(const void *q, const void *k, const void *v, void *o, float *lse, int B, int H, int Hkv,
@@ -316,7 +336,26 @@ int ave_attn_fwd_strided(const void *q, const void *k, const void *v, void *o, f
     st = check_device();
     if (st != AVE_OK) return st;
     return launch_attention(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, causal, scale, 1, 0, nullptr, nullptr, 0, layout,
-                            static_cast<cudaStream_t>(stream));
+                            nullptr, static_cast<cudaStream_t>(stream));
+}
+
+int ave_attn_fwd_varlen(const void *q, const void *k, const void *v, void *o, float *lse, const int *cu_seqlens_q,
+                        const int *cu_seqlens_k, int B, int H, int Hkv, int max_Sq, int max_Sk, int total_q,
+                        int total_k, int D, int causal, float scale, void *stream) {
+    if (!cu_seqlens_q || !cu_seqlens_k) return AVE_ERR_NULL_POINTER;
+    int st = validate(q, k, v, o, lse, B, H, Hkv, max_Sq, max_Sk, D, scale);
+    if (st >= 0) return st;
+    if (total_q <= 0 || total_k <= 0 || total_q >= (1 << 30) || total_k >= (1 << 30)) return AVE_ERR_BAD_SHAPE;
+    if (max_Sq > total_q || max_Sk > total_k) return AVE_ERR_BAD_SHAPE;
+    st = validate_ptrs_and_scale(q, k, v, o, lse, scale);
+    if (st != AVE_OK) return st;
+    if ((reinterpret_cast<uintptr_t>(cu_seqlens_q) | reinterpret_cast<uintptr_t>(cu_seqlens_k)) & 3u)
+        return AVE_ERR_MISALIGNED;
+    st = check_device();
+    if (st != AVE_OK) return st;
+    const VarlenArgs vl{cu_seqlens_q, cu_seqlens_k, total_q, total_k};
+    return launch_attention(q, k, v, o, lse, B, H, Hkv, max_Sq, max_Sk, D, causal, scale, 1, 0, nullptr, nullptr, 0,
+                            nullptr, &vl, static_cast<cudaStream_t>(stream));
 }
 
 size_t ave_attn_host_workspace_bytes(int B, int H, int Hkv, int Sq, int Sk, int D) {

@@ -26,7 +26,7 @@ def declared_functions():
 
 def test_header_declares_the_expected_entry_points():
     names = declared_functions()
-    for n in ("ave_attn_fwd", "ave_attn_fwd_strided", "ave_attn_fwd_host", "ave_attn_host_workspace_bytes", "ave_attn_device_status",
+    for n in ("ave_attn_fwd", "ave_attn_fwd_strided", "ave_attn_fwd_varlen", "ave_attn_fwd_host", "ave_attn_host_workspace_bytes", "ave_attn_device_status",
               "ave_attn_fwd_splitkv", "ave_attn_splitkv_workspace_bytes",
               "ave_attn_launch_count", "ave_attn_strerror", "ave_attn_version", "ave_attn_last_cuda_error"):
         assert n in names
