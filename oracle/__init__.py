@@ -52,6 +52,10 @@ def _load():
             lib.ave_oracle_attn_rows.restype = ctypes.c_int
             lib.ave_oracle_bruteforce.argtypes = [u16p, u16p, u16p, f64p, f64p] + dims
             lib.ave_oracle_bruteforce.restype = ctypes.c_int
+            lib.ave_oracle_gemm_tn.argtypes = [u16p, u16p, f64p] + [ctypes.c_int] * 3
+            lib.ave_oracle_gemm_tn.restype = ctypes.c_int
+            lib.ave_oracle_gemm_tn_entries.argtypes = [u16p, u16p, i64p, ctypes.c_int64, f64p] + [ctypes.c_int] * 3
+            lib.ave_oracle_gemm_tn_entries.restype = ctypes.c_int
             lib.ave_oracle_threads.argtypes = []
             lib.ave_oracle_threads.restype = ctypes.c_int
             _lib = lib
@@ -137,3 +141,35 @@ def bruteforce(q, k, v, causal: bool, scale: float):
     if rc != 0:
         raise ValueError("ave_oracle_bruteforce rejected its arguments (rc=%d)" % rc)
     return o, lse
+
+
+def gemm_tn(a, b):
+    """C [M, N] = A [M, K] . B [N, K]^T in float64 (plain definition)."""
+    ab, bb = _bits(a), _bits(b)
+    if ab.ndim != 2 or bb.ndim != 2 or ab.shape[1] != bb.shape[1]:
+        raise ValueError("a must be [M, K] and b [N, K]")
+    M, K = ab.shape
+    N = bb.shape[0]
+    c = np.empty((M, N), np.float64)
+    rc = _load().ave_oracle_gemm_tn(_ptr(ab, ctypes.c_uint16), _ptr(bb, ctypes.c_uint16), _ptr(c, ctypes.c_double),
+                                    M, N, K)
+    if rc != 0:
+        raise ValueError("ave_oracle_gemm_tn rejected its arguments (rc=%d)" % rc)
+    return c
+
+
+def gemm_tn_entries(a, b, idx):
+    """Oracle values of selected entries; ``idx`` is an [n, 2] array of (i, j)."""
+    ab, bb = _bits(a), _bits(b)
+    if ab.ndim != 2 or bb.ndim != 2 or ab.shape[1] != bb.shape[1]:
+        raise ValueError("a must be [M, K] and b [N, K]")
+    M, K = ab.shape
+    N = bb.shape[0]
+    idx = np.ascontiguousarray(np.asarray(idx, dtype=np.int64).reshape(-1, 2))
+    out = np.empty((idx.shape[0],), np.float64)
+    rc = _load().ave_oracle_gemm_tn_entries(_ptr(ab, ctypes.c_uint16), _ptr(bb, ctypes.c_uint16),
+                                            _ptr(idx, ctypes.c_int64), idx.shape[0], _ptr(out, ctypes.c_double),
+                                            M, N, K)
+    if rc != 0:
+        raise ValueError("ave_oracle_gemm_tn_entries rejected its arguments (rc=%d)" % rc)
+    return out

@@ -213,3 +213,40 @@ int ave_oracle_bruteforce(const uint16_t *q, const uint16_t *k, const uint16_t *
             }
     return 0;
 }
+
+
+/* ------------------------------------------------------------------ GEMM
+ * C[i, j] = sum_k A[i, k] * B[j, k], the plain definition of the matrix product
+ * the paper's GEMM workload computes (Section 9: square bf16 matrices), with
+ * both operands stored with the reduction index contiguous.  fp64 throughout;
+ * rows of C are distributed over OpenMP threads. */
+int ave_oracle_gemm_tn(const uint16_t *a, const uint16_t *b, double *c, int M, int N, int K) {
+    if (!a || !b || !c || M <= 0 || N <= 0 || K <= 0) return 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < M; ++i) {
+        for (int64_t j = 0; j < N; ++j) {
+            double acc = 0.0;
+            for (int64_t k = 0; k < K; ++k)
+                acc += bf16_to_double(a[i * K + k]) * bf16_to_double(b[j * K + k]);
+            c[i * N + j] = acc;
+        }
+    }
+    return 0;
+}
+
+/* The same definition for `n` selected entries: idx[2*e+0..1] = (i, j), out[e] = C[i, j]. */
+int ave_oracle_gemm_tn_entries(const uint16_t *a, const uint16_t *b, const int64_t *idx, int64_t n, double *out,
+                               int M, int N, int K) {
+    if (!a || !b || !idx || !out || M <= 0 || N <= 0 || K <= 0 || n < 0) return 1;
+    for (int64_t e = 0; e < n; ++e)
+        if (idx[2 * e] < 0 || idx[2 * e] >= M || idx[2 * e + 1] < 0 || idx[2 * e + 1] >= N) return 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t e = 0; e < n; ++e) {
+        const int64_t i = idx[2 * e], j = idx[2 * e + 1];
+        double acc = 0.0;
+        for (int64_t k = 0; k < K; ++k)
+            acc += bf16_to_double(a[i * K + k]) * bf16_to_double(b[j * K + k]);
+        out[e] = acc;
+    }
+    return 0;
+}

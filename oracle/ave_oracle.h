@@ -1,5 +1,6 @@
 /*
- * CPU oracle for scaled-dot-product attention forward with log-sum-exp.
+ * CPU oracle for scaled-dot-product attention forward with log-sum-exp
+ * (and, at the end of this header, for the dense matrix product).
  *
  * TEST INFRASTRUCTURE ONLY.  This is the slow, plain, fp64 statement of what
  * the attention forward pass computes.  It exists so that the tests, the smoke
@@ -66,6 +67,19 @@ int ave_oracle_bruteforce(const uint16_t *q, const uint16_t *k, const uint16_t *
                           double *o, double *lse,
                           int B, int H, int Hkv, int Sq, int Sk, int D,
                           int causal, float scale);
+
+/* Matrix product (the paper's GEMM workload, Section 9: square bf16 matrices), plain
+ * definition in fp64:  C[i, j] = sum_k A[i, k] * B[j, k].
+ *   a bf16 bit patterns [M, K], b bf16 bit patterns [N, K], c double [M, N], all row-major.
+ * Pins (tests/test_oracle_pins.py): a hand-computed 2x3 by 3x2 product that a transposed
+ * operand breaks, B = identity, all-ones operands (every entry K), bilinearity under
+ * exact power-of-two scaling, and numpy's fp64 matmul on ragged sizes.
+ * Returns 0, or 1 on a bad argument. */
+int ave_oracle_gemm_tn(const uint16_t *a, const uint16_t *b, double *c, int M, int N, int K);
+
+/* The same definition for n selected entries: idx[2*e+0..1] = (i, j), out[e] = C[i, j]. */
+int ave_oracle_gemm_tn_entries(const uint16_t *a, const uint16_t *b, const int64_t *idx, int64_t n, double *out,
+                               int M, int N, int K);
 
 /* Number of OpenMP threads ave_oracle_attn_fwd / _rows will use. */
 int ave_oracle_threads(void);

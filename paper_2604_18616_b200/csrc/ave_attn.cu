@@ -2,6 +2,7 @@
 // TMA tensor-map encoding, kernel selection and launch.  See include/ave_attn.h
 // for the contract of every exported function.
 #include "../../include/ave_attn.h"
+#include "../../include/ave_gemm.h"
 
 #include <atomic>
 #include <cmath>
@@ -13,6 +14,7 @@
 #include <cuda_bf16.h>
 
 #include "attn_fwd_ws.cuh"
+#include "gemm_bf16.cuh"
 
 // Scratch of ave_attn_fwd_splitkv_static: part of the device image, so every GPU that loads the
 // library holds it until exit.  In host code this name is only a handle for
@@ -298,6 +300,52 @@ int run_splitkv(const void *q, const void *k, const void *v, void *o, float *lse
     return AVE_OK;
 }
 
+
+// C[M, N] = A[M, K] * B[N, K]^T: tensor maps of the three matrices, tile order, persistent launch.
+int launch_gemm_tn(const void *a, const void *b, void *c, int M, int N, int K, cudaStream_t s) {
+    using Cfg = ave::GemmCfg;
+    CUtensorMap ta, tb, tc;
+    const Strides sa{(long long)M * K, (long long)M * K, (long long)K};
+    const Strides sb{(long long)N * K, (long long)N * K, (long long)K};
+    const Strides sc{(long long)M * N, (long long)M * N, (long long)N};
+    if (!encode_map(&ta, a, K, M, 1, 1, sa, Cfg::kTileM)) return AVE_ERR_CUDA;
+    if (!encode_map(&tb, b, K, N, 1, 1, sb, Cfg::kTileN)) return AVE_ERR_CUDA;
+    if (!encode_map(&tc, c, N, M, 1, 1, sc, Cfg::kOutBoxRows)) return AVE_ERR_CUDA;
+    ave::GemmParams p;
+    p.M = M;
+    p.N = N;
+    p.K = K;
+    p.tiles_m = (M + Cfg::kTileM - 1) / Cfg::kTileM;
+    p.tiles_n = (N + Cfg::kTileN - 1) / Cfg::kTileN;
+    p.group_m = 8;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess || sms <= 0) {
+        t_last_cuda_error = int(e);
+        return AVE_ERR_CUDA;
+    }
+    static std::atomic<bool> configured{false};
+    if (!configured.load(std::memory_order_acquire)) {
+        e = cudaFuncSetAttribute(ave::gemm_bf16_tn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
+        if (e != cudaSuccess) {
+            t_last_cuda_error = int(e);
+            return AVE_ERR_CUDA;
+        }
+        configured.store(true, std::memory_order_release);
+    }
+    const long long n_tiles = (long long)p.tiles_m * p.tiles_n;
+    const unsigned grid = unsigned(n_tiles < sms ? n_tiles : sms);
+    ave::gemm_bf16_tn_kernel<<<dim3(grid), dim3(Cfg::kThreads), Cfg::kSmemBytes, s>>>(ta, tb, tc, p);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        t_last_cuda_error = int(e);
+        return AVE_ERR_CUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return AVE_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -521,6 +569,20 @@ int ave_attn_trace_read(long long *out) {
     return e == cudaSuccess ? AVE_OK : AVE_ERR_CUDA;
 }
 #endif
+
+int ave_gemm_bf16_tn(const void *a, const void *b, void *c, int M, int N, int K, void *stream) {
+    if (!a || !b || !c) return AVE_ERR_NULL_POINTER;
+    if (M <= 0 || N <= 0 || K <= 0) return AVE_ERR_BAD_SHAPE;
+    const long long lim = 1ll << 40;
+    if ((long long)M * K >= lim || (long long)N * K >= lim || (long long)M * N >= lim) return AVE_ERR_BAD_SHAPE;
+    if ((long long)((M + 127) / 128) * ((N + 255) / 256) >= (1ll << 31)) return AVE_ERR_BAD_SHAPE;
+    if ((K & 7) || (N & 7)) return AVE_ERR_MISALIGNED;
+    if ((reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b) | reinterpret_cast<uintptr_t>(c)) & 15u)
+        return AVE_ERR_MISALIGNED;
+    int st = check_device();
+    if (st != AVE_OK) return st;
+    return launch_gemm_tn(a, b, c, M, N, K, static_cast<cudaStream_t>(stream));
+}
 
 int ave_attn_last_cuda_error(void) { return t_last_cuda_error; }
 

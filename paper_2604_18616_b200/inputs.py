@@ -147,3 +147,13 @@ def sample_rows(w: Workload, n_random: int, seed: int = 12345, tile: int = 128):
         ri = torch.randint(0, w.Sq, (n_random,), generator=g)
         rows += list(zip(rb.tolist(), rh.tolist(), ri.tolist()))
     return rows
+
+
+def make_gemm_inputs(M: int, N: int, K: int, seed: int):
+    """A [M, K] and B [N, K] for the matrix-product workload (the paper's Section 9: bf16 matrices
+    with normally distributed entries): one CPU generator draws fp32 A, then B, N(0,1), rounded to bf16."""
+    g = torch.Generator(device="cpu")
+    g.manual_seed(seed)
+    a = torch.randn((M, K), generator=g, dtype=torch.float32).to(torch.bfloat16)
+    b = torch.randn((N, K), generator=g, dtype=torch.float32).to(torch.bfloat16)
+    return a, b

@@ -19,16 +19,23 @@ def lib():
 
 
 def declared_functions():
-    text = open(os.path.join(ROOT, "include", "ave_attn.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(ave_attn_\w+)\s*\(", text)))
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for header in sorted(os.listdir(inc)):
+        if not header.endswith(".h"):
+            continue
+        text = open(os.path.join(inc, header)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names.update(re.findall(r"\b(ave_(?:attn|gemm)_\w+)\s*\(", text))
+    return sorted(names)
 
 
 def test_header_declares_the_expected_entry_points():
     names = declared_functions()
     for n in ("ave_attn_fwd", "ave_attn_fwd_strided", "ave_attn_fwd_varlen", "ave_attn_fwd_host", "ave_attn_host_workspace_bytes", "ave_attn_device_status",
               "ave_attn_fwd_splitkv", "ave_attn_splitkv_workspace_bytes",
-              "ave_attn_launch_count", "ave_attn_strerror", "ave_attn_version", "ave_attn_last_cuda_error"):
+              "ave_attn_launch_count", "ave_attn_strerror", "ave_attn_version", "ave_attn_last_cuda_error",
+              "ave_gemm_bf16_tn"):
         assert n in names
 
 
@@ -97,3 +104,18 @@ def test_host_entry_point_validates_workspace(lib):
     assert st == binding.AVE_ERR_WORKSPACE
     st = L.ave_attn_fwd_host(vp(A), vp(A), vp(A), vp(A), vp(A), 1, 2, 2, 128, 128, 64, 0, 1.0, vp(A), 16, vp(0))
     assert st == binding.AVE_ERR_WORKSPACE
+
+
+def test_gemm_validation_before_any_cuda_call(lib):
+    A = 4096  # aligned fake address: validation must reject before dereferencing anything
+    f = binding.ave_gemm_bf16_tn_raw
+    assert f(0, A, A, 128, 256, 64) == binding.AVE_ERR_NULL_POINTER
+    assert f(A, 0, A, 128, 256, 64) == binding.AVE_ERR_NULL_POINTER
+    assert f(A, A, 0, 128, 256, 64) == binding.AVE_ERR_NULL_POINTER
+    assert f(A, A, A, 0, 256, 64) == binding.AVE_ERR_BAD_SHAPE
+    assert f(A, A, A, 128, -8, 64) == binding.AVE_ERR_BAD_SHAPE
+    assert f(A, A, A, 128, 256, 0) == binding.AVE_ERR_BAD_SHAPE
+    assert f(A, A, A, 2 ** 21, 256, 2 ** 21) == binding.AVE_ERR_BAD_SHAPE      # M * K beyond 2^40
+    assert f(A, A, A, 128, 250, 64) == binding.AVE_ERR_MISALIGNED               # N not a multiple of 8
+    assert f(A, A, A, 128, 256, 68) == binding.AVE_ERR_MISALIGNED               # K not a multiple of 8
+    assert f(A + 8, A, A, 128, 256, 64) == binding.AVE_ERR_MISALIGNED

@@ -234,3 +234,40 @@ def test_bad_arguments_are_rejected():
     q, k, v = rand_qkv(0, 1, 3, 2, 4, 4, 4)   # H % Hkv != 0
     with pytest.raises(ValueError):
         oracle.attn_fwd(q, k, v, False, 1.0)
+
+
+# ------------------------------------------------------------------ GEMM oracle pins
+def _bf16(x):
+    return torch.tensor(x, dtype=torch.float32).to(torch.bfloat16)
+
+
+def test_gemm_hand_example_breaks_on_a_transposed_operand():
+    # A (2x3) . B^T with B (2x3):  rows of A dotted with rows of B, by hand
+    a = _bf16([[1, 2, 3], [4, 5, 6]])
+    b = _bf16([[7, 8, 9], [1, 0, -1]])
+    c = oracle.gemm_tn(a, b)
+    assert np.array_equal(c, np.array([[50.0, -2.0], [122.0, -2.0]]))
+
+
+def test_gemm_identity_and_ones():
+    g = torch.Generator().manual_seed(5)
+    a = torch.randn((7, 16), generator=g).to(torch.bfloat16)
+    eye = torch.eye(16).to(torch.bfloat16)
+    assert np.array_equal(oracle.gemm_tn(a, eye), a.double().numpy())
+    ones_a = torch.ones((3, 40)).to(torch.bfloat16)
+    ones_b = torch.ones((5, 40)).to(torch.bfloat16)
+    assert np.array_equal(oracle.gemm_tn(ones_a, ones_b), np.full((3, 5), 40.0))
+
+
+def test_gemm_bilinear_under_exact_scaling_and_matches_numpy():
+    g = torch.Generator().manual_seed(6)
+    a = torch.randn((33, 72), generator=g).to(torch.bfloat16)
+    b = torch.randn((19, 72), generator=g).to(torch.bfloat16)
+    c = oracle.gemm_tn(a, b)
+    a4 = (a.float() * 4).to(torch.bfloat16)      # exact in bf16
+    bh = (b.float() * 0.5).to(torch.bfloat16)
+    np.testing.assert_allclose(oracle.gemm_tn(a4, bh), 2.0 * c, rtol=0, atol=0)
+    ref = a.double().numpy() @ b.double().numpy().T  # the library routine, fp64
+    np.testing.assert_allclose(c, ref, rtol=1e-13, atol=1e-13)
+    idx = np.array([[0, 0], [32, 18], [5, 7]])
+    np.testing.assert_array_equal(oracle.gemm_tn_entries(a, b, idx), c[idx[:, 0], idx[:, 1]])
