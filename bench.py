@@ -30,7 +30,8 @@ DEFAULT_WORKLOAD = "c2_mha_prefill"
 NOMINAL_BF16_TFLOPS = 2250.0          # vendor dense bf16 figure, context only
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu captures summarised under
 # profiles/ (attn_fwd_ws_<workload>_ncu_full.md); null for workloads that were not captured.
-NCU_DRAM_BYTES_PER_LAUNCH = {"c2_mha_prefill": 326.2e6, "c3_gqa_prefill": 276.5e6}
+NCU_DRAM_BYTES_PER_LAUNCH = {"c2_mha_prefill": 326.2e6, "c3_gqa_prefill": 276.5e6,
+                             "c4_long_context": 508.4e6, "c5_wide_noncausal": 1825.0e6}
 FALLBACK_BF16_TFLOPS = 1590.0         # earlier measurement on this machine, used when no measured file exists
 
 
