@@ -4,7 +4,8 @@
   python bench.py --gpus N --steps K --warmup W [--workload NAME] [--impl reference]
 
 One step = one ave_attn_fwd pass over one batch of the named synthetic
-workload.  Rank 0 prints ONE JSON line.  `value` is counted TFLOP/s
+workload (`--workload gemm_n<size>`: one ave_gemm_bf16_tn product of square
+matrices of that size, reported in its own metric).  Rank 0 prints ONE JSON line.  `value` is counted TFLOP/s
 (4*B*H*Sq*Sk*D, halved when causal) over all ranks with inputs resident in
 HBM; `e2e` is the same metric through the host-buffer entry point with the
 host<->device copies inside the timed region; `roofline` relates the kernel's
@@ -297,11 +298,190 @@ def run_ours(args):
     return 0
 
 
+
+# ------------------------------------------------------------------- GEMM workload
+GEMM_METRIC = "gemm TFLOP/s (bf16, 2*M*N*K)"
+
+
+def gemm_size(name):
+    """'gemm_n8192' -> 8192 (square product, the paper's Section 9 GEMM workload)."""
+    n = int(name[len("gemm_n"):])
+    if n <= 0 or n % 8:
+        raise ValueError("gemm_n<size>: size must be a positive multiple of 8")
+    return n
+
+
+def gemm_oracle_sample(a, b, target_seconds):
+    """Time the fp64 oracle on evenly spread entries of C; returns (TFLOP/s, cores, description, seconds)."""
+    import numpy as np
+    import oracle
+    M, K = a.shape
+    N = b.shape[0]
+
+    def entries(n):
+        idx = np.linspace(0, M * N - 1, n).astype(np.int64)
+        return np.stack([idx // N, idx % N], axis=1)
+
+    cores = oracle.threads()
+    probe = entries(max(20000, 2000 * cores))
+    t0 = time.perf_counter()
+    oracle.gemm_tn_entries(a, b, probe)
+    t_probe = time.perf_counter() - t0
+    n = int(min(M * N, max(len(probe), len(probe) * target_seconds / max(t_probe, 1e-6))))
+    t0 = time.perf_counter()
+    oracle.gemm_tn_entries(a, b, entries(n))
+    dt = time.perf_counter() - t0
+    tf = 2.0 * K * n / dt / 1e12
+    desc = "%d of %d entries of C (%dx%dx%d), evenly spread, %.1f s; 2*K flops per entry" % (n, M * N, M, N, K, dt)
+    return tf, cores, desc, dt
+
+
+def run_gemm_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from paper_2604_18616_b200 import inputs
+    n = gemm_size(args.workload)
+    a, b = inputs.make_gemm_inputs(n, n, n, seed=20)
+    steps = max(1, min(args.steps, 5))
+    warm = max(0, min(args.warmup, 1))
+    per_step = max(2.0, min(args.cpu_seconds, 60.0 / (steps + warm)))
+    for _ in range(warm):
+        gemm_oracle_sample(a, b, per_step)
+    tfs, total, desc, cores = [], 0.0, "", 1
+    for _ in range(steps):
+        tf, cores, desc, dt = gemm_oracle_sample(a, b, per_step)
+        tfs.append(tf)
+        total += dt
+    value = sum(tfs) / len(tfs)
+    print(json.dumps({
+        "impl": "reference", "metric": GEMM_METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": warm, "ms_per_step": 1e3 * total / steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "M": n, "N": n, "K": n,
+                   "note": "each step is a bounded sample of the entries of C"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+    return 0
+
+
+def run_gemm(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2604_18616_b200 import binding, inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the GEMM path has no CPU fallback")
+    binding.lib()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    n = gemm_size(args.workload)
+    a, b = inputs.make_gemm_inputs(n, n, n, seed=20 + 1000 * rank)   # an independent product per rank
+    ad, bd = a.to(dev), b.to(dev)
+    c = torch.empty((n, n), dtype=torch.bfloat16, device=dev)
+    flops = 2.0 * n * n * n
+    stream = torch.cuda.current_stream()
+
+    def step():
+        binding.ave_gemm_bf16_tn(ad, bd, c, stream=stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    n0 = binding.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local_rank) as clocks:
+        barrier()
+        ev0.record(stream)
+        for _ in range(args.steps):
+            step()
+        ev1.record(stream)
+        barrier()
+    ms = ev0.elapsed_time(ev1)
+    launches = binding.launch_count() - n0
+    st, raw = binding.device_status()
+    if st != binding.AVE_OK:
+        raise RuntimeError("device status %d (raw %#x) after the timed region" % (st, raw))
+
+    # ---- end to end: pinned host operands in, host result out, copies inside the timed region
+    e2e_steps = max(1, args.e2e_steps)
+    ah, bh = a.pin_memory(), b.pin_memory()
+    ch = torch.empty((n, n), dtype=torch.bfloat16).pin_memory()
+
+    def e2e_step():
+        ad.copy_(ah, non_blocking=True)
+        bd.copy_(bh, non_blocking=True)
+        binding.ave_gemm_bf16_tn(ad, bd, c, stream=stream)
+        ch.copy_(c, non_blocking=True)
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+
+    t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_max, e2e_ms_max = t.tolist()
+    if rank == 0:
+        peak, peak_kind, peaks = measured_peak()
+        sustained = float(peaks["bf16_tflops_sustained"]) if peaks and "bf16_tflops_sustained" in peaks else None
+        ms_per_step = ms_max / args.steps
+        kernel_tf = flops / ((ms / args.steps) * 1e-3) / 1e12
+        line = {
+            "metric": GEMM_METRIC, "value": world * flops / (ms_per_step * 1e-3) / 1e12, "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": args.workload, "M": n, "N": n, "K": n, "layout": "A [M,K], B [N,K], C [M,N] row-major",
+                       "parallelism": "dp%d (independent products)" % world,
+                       "l2": "A+B+C = %.0f MiB per step%s" % (3 * n * n * 2 / 2 ** 20,
+                                                             " exceed the 126 MB L2; no explicit flush" if 3 * n * n * 2 > 126e6
+                                                             else " fit in L2 (no flush): a cache-resident case")},
+            "clocks": clocks.summary(),
+            "e2e": {"value": world * flops / (e2e_ms_max / e2e_steps * 1e-3) / 1e12, "unit": UNIT,
+                    "h2d_bytes_per_step": 2 * n * n * 2, "d2h_bytes_per_step": n * n * 2, "steps": e2e_steps},
+            "gpu_launches": int(launches),
+            "roofline": {"bound": "tensor", "achieved": kernel_tf, "peak": peak, "unit": "TFLOP/s",
+                         "frac": kernel_tf / peak, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(args.workload),
+                         "traffic_unit": "bytes per launch (ncu dram read+write)",
+                         "algorithmic_hbm_bytes": 3 * n * n * 2, "peak_kind": peak_kind,
+                         "frac_of_nominal_2250": kernel_tf / NOMINAL_BF16_TFLOPS, "peak_sustained": sustained,
+                         "frac_of_sustained": (kernel_tf / sustained) if sustained else None,
+                         "flops_per_launch": flops, "kernel_us": 1e3 * ms / args.steps},
+        }
+        if not args.no_cpu_baseline and world == 1:
+            tf, cores, desc, _ = gemm_oracle_sample(a, b, args.cpu_seconds)
+            line["cpu_baseline"] = {"value": tf, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
 def main():
     args = parse_args()
+    is_gemm = args.workload.startswith("gemm_n")
     if args.impl == "reference":
-        return run_reference(args)
-    return run_ours(args)
+        return run_gemm_reference(args) if is_gemm else run_reference(args)
+    return run_gemm(args) if is_gemm else run_ours(args)
 
 
 if __name__ == "__main__":
