@@ -569,8 +569,13 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const uint32_t tS = tmem + (t ? Cfg::kColS1 : Cfg::kColS0) + lane_sel;
         const uint32_t tO = tmem + (t ? Cfg::kColO1 : Cfg::kColO0) + lane_sel;
         const uint32_t sO = sStage + t * Cfg::kStageOBytes + wq * (Cfg::kOutBoxRows * 128);  // this warp's 32 rows
-        const float sl2 = p.scale_log2;
-        const bool neg = sl2 < 0.f;
+        // The softmax works with a positive scale only, which keeps one maximum-then-exponentiate
+        // code path (the kernel's code has to stay within the instruction cache): a negative scale
+        // negates the scores in TMEM first and then uses |scale|; a zero scale (all visible keys
+        // weigh the same) is replaced by 2^-100, under which every visible score still rounds to
+        // an exponent of 0 while a masked one stays -inf.
+        const bool neg = p.scale_log2 < 0.f;
+        const float sl2 = (p.scale_log2 == 0.f) ? 7.888609052210118e-31f : fabsf(p.scale_log2);
         const bool tracer = (r == 0);
         uint32_t ns = 0;             // S_t tiles consumed so far (phase of bar_s[t])
         uint32_t n_out = 0;          // finished O_t accumulators taken so far (phase of bar_o[t])
@@ -627,6 +632,18 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     ++ns;
                     if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 1);
                     tc_fence_after();
+                    if (neg) {  // S_t <- -S_t in place (rare path, kept small)
+#pragma unroll 1
+                        for (int c = 0; c < 8; ++c) {
+                            uint32_t sc[16];
+                            tmem_ld_x16(tS + c * 16, sc);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) sc[e] ^= 0x80000000u;
+                            tmem_st_x16(tS + c * 16, sc);
+                        }
+                        tmem_wait_st();
+                    }
                     uint32_t sraw[4][32];
 #pragma unroll
                     for (int c = 0; c < 4; ++c) tmem_ld_x32(tS + c * 32, sraw[c]);
@@ -642,40 +659,25 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         if (CAUSAL) lim = min(lim, i + off - j0);
                     }
 
-                    // ---- row extreme of the raw scores (maximum of scale*s is at max s, or min s if scale < 0)
-                    // With a positive scale a masked score is simply replaced by -inf: it then drops out
-                    // of the maximum and its probability exp2(-inf) is exactly 0.  Zero and negative
-                    // scales (where -inf * scale is not -inf) take the explicit, slower path below.
-                    const bool generic = !(sl2 > 0.f);
-                    if (need_mask && !generic) {
+                    // ---- row maximum of the raw scores.  A masked score is simply replaced by -inf: it then
+                    // drops out of the maximum and its probability exp2(-inf) is exactly 0.
+                    if (need_mask) {
 #pragma unroll
                         for (int c = 0; c < 128; ++c)
                             sraw[c >> 5][c & 31] = (c <= lim) ? sraw[c >> 5][c & 31] : 0xff800000u;
                     }
-                    // Row extreme of the (masked) raw scores, as scale*log2(e)*s; -inf if nothing is visible.
+                    // Row maximum of the (masked) raw scores, as scale*log2(e)*s; -inf if nothing is visible.
                     auto tile_max = [&]() -> float {
-                        float ext;
-                        if (!generic) {
-                            float e0 = -INFINITY, e1 = -INFINITY, e2 = -INFINITY, e3 = -INFINITY;
+                        float e0 = -INFINITY, e1 = -INFINITY, e2 = -INFINITY, e3 = -INFINITY;
 #pragma unroll
-                            for (int c = 0; c < 32; c += 2) {
-                                e0 = max3(e0, __uint_as_float(sraw[0][c]), __uint_as_float(sraw[0][c + 1]));
-                                e1 = max3(e1, __uint_as_float(sraw[1][c]), __uint_as_float(sraw[1][c + 1]));
-                                e2 = max3(e2, __uint_as_float(sraw[2][c]), __uint_as_float(sraw[2][c + 1]));
-                                e3 = max3(e3, __uint_as_float(sraw[3][c]), __uint_as_float(sraw[3][c + 1]));
-                            }
-                            ext = fmaxf(fmaxf(e0, e1), fmaxf(e2, e3));
-                        } else {
-                            ext = neg ? INFINITY : -INFINITY;
-#pragma unroll
-                            for (int c = 0; c < 128; ++c) {
-                                const float s = __uint_as_float(sraw[c >> 5][c & 31]);
-                                const bool vis = !need_mask || (c <= lim);
-                                if (neg) ext = vis ? fminf(ext, s) : ext;
-                                else     ext = vis ? fmaxf(ext, s) : ext;
-                            }
+                        for (int c = 0; c < 32; c += 2) {
+                            e0 = max3(e0, __uint_as_float(sraw[0][c]), __uint_as_float(sraw[0][c + 1]));
+                            e1 = max3(e1, __uint_as_float(sraw[1][c]), __uint_as_float(sraw[1][c + 1]));
+                            e2 = max3(e2, __uint_as_float(sraw[2][c]), __uint_as_float(sraw[2][c + 1]));
+                            e3 = max3(e3, __uint_as_float(sraw[3][c]), __uint_as_float(sraw[3][c + 1]));
                         }
-                        return (fabsf(ext) == INFINITY) ? -INFINITY : ext * sl2;
+                        const float ext = fmaxf(fmaxf(e0, e1), fmaxf(e2, e3));
+                        return (ext == -INFINITY) ? -INFINITY : ext * sl2;
                     };
                     // p = exp2(scale*log2e*s - m) for the whole row: P -> bf16 pairs into TMEM over the
                     // first 64 columns of S_t; returns the row sum of the fp32 probabilities.
@@ -697,10 +699,6 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                                     pr.x = ex2_approx(x.x);
                                     pr.y = ex2_approx(x.y);
                                 }
-                                if (need_mask && generic) {
-                                    pr.x = (cc * 32 + e <= lim) ? pr.x : 0.f;
-                                    pr.y = (cc * 32 + e + 1 <= lim) ? pr.y : 0.f;
-                                }
                                 if (e & 2) acc1 = __fadd2_rn(acc1, pr);  // fp32 probabilities, before rounding to bf16
                                 else       acc0 = __fadd2_rn(acc0, pr);
                                 pk[e >> 1] = pack_bf16x2(pr.x, pr.y);
@@ -711,7 +709,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     };
                     // O <- alpha * O.  S_t(j) ready implies P_t V_{j-1} has finished (in-order tensor pipe).
                     auto rescale_o = [&](float alpha) {
-#pragma unroll
+#pragma unroll 1
                         for (int c = 0; c < D / 32; ++c) {
                             uint32_t oc[32];
                             tmem_ld_x32(tO + c * 32, oc);
