@@ -37,8 +37,10 @@ struct FwdParams {
     int Sq, Sk;       // sequence lengths
     int BH;           // B * H
     int n_qblk;       // work tiles (blocks of 256 query rows) per (b, h)
-    int total_blocks; // n_qblk * BH = grid size
-    int heads_per_group;  // (b, h) pairs whose work tiles are launched together (their K/V share L2)
+    int total_blocks; // grid size: n_qblk * n_units * n_splits
+    int pair_heads;   // != 0: a work tile is 128 query rows of two neighbouring query heads of one key/value head
+    int n_units;      // BH, or BH / 2 when heads are paired
+    int heads_per_group;  // units ((b, h) pairs, or pairs of heads) whose work tiles are launched together (their K/V share L2)
     float scale_log2; // scale * log2(e)
     int causal_off;   // key j is visible to query i iff j <= i + causal_off (Sk - Sq of the whole problem)
     // Split-KV launches only: the keys are cut into n_splits ranges of keys_per_split (a multiple of

@@ -86,6 +86,8 @@ struct WorkTileBase {
     int b, h;    // batch and query head
     int g;       // h / (H / Hkv): key/value head (Fig. 1: idx_h / gqa)
     int q0;      // first query row
+    int dq, dh;  // sub-tile 1 relative to sub-tile 0: rows further down (BM, same head) or, in launches that
+                 // pair heads, the next query head of the same key/value head (same rows)
     int n0, n1;  // key tiles the two sub-tiles visit (n1 >= n0)
 };
 template <bool SPLIT>
@@ -155,18 +157,25 @@ __device__ __forceinline__ TileOf<SPLIT, VARLEN> decode_tile(int id, const FwdPa
         w.k_begin = k_begin = min(p.Sk, w.split * p.keys_per_split);
         w.k_end = k_end = min(p.Sk, w.k_begin + p.keys_per_split);
     }
+    // A unit is a (batch, head) pair or, when heads are paired, two neighbouring query heads of one
+    // key/value head: the two sub-tiles then take the same 128 query rows of the two heads, so that in a
+    // causal launch both visit the same key tiles and reach the diagonal, and the next tile, together.
+    const bool paired = !SPLIT && !VARLEN && p.pair_heads != 0;
     const int per_group = p.heads_per_group * p.n_qblk;
     const int grp = id / per_group;
     const int rem = id - grp * per_group;
-    const int bh0 = grp * p.heads_per_group;
-    const int hg = min(p.heads_per_group, p.BH - bh0);
+    const int u0 = grp * p.heads_per_group;
+    const int hg = min(p.heads_per_group, p.n_units - u0);
     const int rank = rem / hg;
-    w.bh = bh0 + (rem - rank * hg);
+    const int unit = u0 + (rem - rank * hg);
+    w.bh = paired ? 2 * unit : unit;
+    w.dq = paired ? 0 : BM;
+    w.dh = paired ? 1 : 0;
     const int qb = CAUSAL ? (p.n_qblk - 1 - rank) : rank;
     w.b = w.bh / p.H;
     w.h = w.bh - w.b * p.H;
     w.g = w.h / (p.H / p.Hkv);
-    w.q0 = qb * 2 * BM;
+    w.q0 = qb * (paired ? BM : 2 * BM);
     if constexpr (SPLIT) {
         w.n0 = kv_tiles_for<CAUSAL>(query_pos_hi(w.q0, p.rows_per_head), p.causal_off, k_begin, k_end);
         w.n1 = max(w.n0, kv_tiles_for<CAUSAL>(query_pos_hi(w.q0 + BM, p.rows_per_head), p.causal_off, k_begin, k_end));
@@ -181,7 +190,7 @@ __device__ __forceinline__ TileOf<SPLIT, VARLEN> decode_tile(int id, const FwdPa
         w.n1 = max(w.n0, w.n1);
     } else {
         w.n0 = kv_tiles_whole<CAUSAL>(w.q0, p.Sq, p.Sk);
-        w.n1 = kv_tiles_whole<CAUSAL>(w.q0 + BM, p.Sq, p.Sk);
+        w.n1 = kv_tiles_whole<CAUSAL>(w.q0 + w.dq, p.Sq, p.Sk);
     }
     return w;
 }
@@ -371,7 +380,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         mbar_arrive_expect_tx(bar, Cfg::kTileBytes);
                         for (int x = 0; x < Cfg::kBoxes; ++x)  // the tensor maps are {D, rows, heads, batch}
                             tma_load_4d(sQ + t * Cfg::kTileBytes + x * Cfg::kBoxBytes, &tm_q, bar, x * 64,
-                                        q_base_of(w) + w.q0 + t * BM, w.h, batch_coord(w));
+                                        q_base_of(w) + w.q0 + t * w.dq, w.h + t * w.dh, batch_coord(w));
                     }
                 };
                 try_load_q(0, false);
@@ -584,11 +593,13 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 
         int id = blockIdx.x;
         for (int n = 0; id >= 0 && ok; ++n) {
-            const TileOf<SPLIT, VARLEN> w = decode_tile<CAUSAL, SPLIT, VARLEN>(id, p);
+            TileOf<SPLIT, VARLEN> w = decode_tile<CAUSAL, SPLIT, VARLEN>(id, p);
+            w.h += t * w.dh;                           // this sub-tile's query head (head-paired launches)
+            w.bh += t * w.dh;
             const int bh = w.bh;
             const int sq = seq_q(w, p);                // query rows of this tile's sequence
             const int off = SPLIT ? p.causal_off : seq_k(w, p) - sq;
-            const int i0 = w.q0 + t * BM;
+            const int i0 = w.q0 + t * w.dq;
             const int i = i0 + r;                     // query row
             const int n_t = t ? w.n1 : w.n0;
 

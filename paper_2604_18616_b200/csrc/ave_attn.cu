@@ -190,27 +190,33 @@ int launch_attention(const void *q, const void *k, const void *v, void *o, float
     p.Sq = Sq;
     p.Sk = Sk;
     p.BH = B * H;
-    p.n_qblk = (Sq + 2 * ave::BM - 1) / (2 * ave::BM);
+    const int G = H / Hkv;
+    // Causal launches with an even number of query heads per key/value head give the two sub-tiles of a work
+    // tile the same 128 query rows of two neighbouring heads instead of 256 rows of one head: both then visit
+    // the same key tiles and finish together, where otherwise sub-tile 1 works through its diagonal step alone.
+    p.pair_heads = (causal && !split && !varlen && rows_per_head == 0 && G % 2 == 0) ? 1 : 0;
+    p.n_units = p.pair_heads ? p.BH / 2 : p.BH;
+    const int rows_per_tile = p.pair_heads ? ave::BM : 2 * ave::BM;
+    p.n_qblk = (Sq + rows_per_tile - 1) / rows_per_tile;
     p.causal_off = Sk - (rows_per_head > 0 ? rows_per_head : Sq);
     p.rows_per_head = rows_per_head;
     p.n_splits = split ? n_splits : 1;
     p.keys_per_split = split ? keys_per_split : Sk;
     p.o_partial = o_partial;
     p.lse_partial = lse_partial;
-    const long long total = (long long)p.n_qblk * p.BH * p.n_splits;
+    const long long total = (long long)p.n_qblk * p.n_units * p.n_splits;
     if (total >= (1ll << 31)) return AVE_ERR_BAD_SHAPE;
     p.total_blocks = int(total);
     {
-        // Launch (b, h) pairs in groups whose K and V together stay within a slice of L2,
+        // Launch units in groups whose K and V together stay within a slice of L2,
         // whole key/value heads at a time.
         const long long kv_bytes_per_kv_head = 2ll * Sk * D * 2;
-        const int G = H / Hkv;
         const long long budget = 64ll << 20;
         long long kv_heads = budget / kv_bytes_per_kv_head;
         if (kv_heads < 1) kv_heads = 1;
-        long long hpg = kv_heads * G;
-        if (hpg > p.BH) hpg = p.BH;
-        p.heads_per_group = int(hpg);
+        long long upg = kv_heads * G / (p.pair_heads ? 2 : 1);
+        if (upg > p.n_units) upg = p.n_units;
+        p.heads_per_group = int(upg);
     }
     p.scale_log2 = scale * 1.4426950408889634f;
 
