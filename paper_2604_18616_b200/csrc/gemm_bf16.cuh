@@ -2,7 +2,8 @@
 // in TMEM, bf16 result.  (The paper's first evaluated kernel family, Section 9:
 // square bf16 matrices with normally distributed entries.)
 //
-// Persistent CTAs, one per SM, each walking output tiles of 128 x 256 in a
+// Persistent CTAs, one per SM, each walking output tiles of 128 x 256 (128 x 128
+// for small products) in a
 // static order.  Inside a tile the K dimension is streamed in slices of 64
 // through a ring of shared-memory stages filled by TMA; one thread issues
 // M128 x N256 x K16 tcgen05 MMAs into one of two TMEM accumulators, so the
@@ -23,17 +24,21 @@
 
 namespace ave {
 
+// TN = 256 is the tile for large products; TN = 128 halves the tile for products with fewer 128 x 256
+// tiles than SMs, where more, shorter tiles finish earlier.
+template <int TN>
 struct GemmCfg {
+    static_assert(TN == 128 || TN == 256, "tile widths the kernel is instantiated for");
     static constexpr int kThreads = 256;
-    static constexpr int kTileM = 128, kTileN = 256, kSliceK = 64;
-    static constexpr int kStages = 4;
+    static constexpr int kTileM = 128, kTileN = TN, kSliceK = 64;
+    static constexpr int kStages = (TN == 256) ? 4 : 6;
     static constexpr int kABytes = kTileM * kSliceK * 2;          // 16 KB
     static constexpr int kBBytes = kTileN * kSliceK * 2;          // 32 KB
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kOutBoxRows = 32;                        // each epilogue warp stores its own 32 rows
     static constexpr int kStageCBytes = 4 * kOutBoxRows * 128;    // C staging: 32 rows x 64 columns per epilogue warp
     static constexpr int kSmemBytes = kStages * kStageBytes + kStageCBytes + 1024;
-    static constexpr uint32_t kTmemCols = 512;                    // two accumulators of 256 columns
+    static constexpr uint32_t kTmemCols = 2 * TN;                 // two accumulators of TN columns
 };
 
 struct GemmParams {
@@ -54,10 +59,11 @@ __device__ __forceinline__ void gemm_tile_coords(int id, const GemmParams &p, in
     bm = m0 + (rem - bn * gm);
 }
 
+template <int TN>
 __global__ void __launch_bounds__(256, 1)
 gemm_bf16_tn_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                     const __grid_constant__ CUtensorMap tm_c, const GemmParams p) {
-    using Cfg = GemmCfg;
+    using Cfg = GemmCfg<TN>;
     constexpr int NS = Cfg::kStages;
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[NS], bar_empty[NS], bar_acc_full[2], bar_acc_empty[2], bar_drain;
