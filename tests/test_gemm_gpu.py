@@ -40,6 +40,8 @@ def run_gemm(a, b, guard=64):
     (300, 1000, 200),      # ragged, several tiles
     (129, 8, 4104),        # long reduction with a ragged last slice
     (2048, 2048, 2048),    # more tiles than SMs: CTAs walk several tiles, both accumulators in use
+    (2100, 2312, 264),     # the 128 x 256 tile kernel (170 tiles) with ragged edges in every dimension
+    (1024, 1024, 1024),    # the 128 x 128 tile kernel, 64 tiles
 ])
 def test_gemm_matches_oracle(M, N, K):
     a, b = inputs.make_gemm_inputs(M, N, K, seed=100 + M + N + K)
