@@ -37,6 +37,14 @@ extern "C" {
  */
 int ave_gemm_bf16_tn(const void *a, const void *b, void *c, int M, int N, int K, void *stream);
 
+/*
+ * The same product with B stored the other way round, the plain C = A B of the paper's Section 9 workload:
+ *   C[i, j] = sum_{k < K} A[i, k] * B[k, j]
+ * a: bf16 [M, K] row-major.  b: bf16 [K, N] row-major.  c: bf16 [M, N] row-major.  Same limits, alignment
+ * rules, errors and arithmetic as ave_gemm_bf16_tn; B is read in place (no transposition pass).
+ */
+int ave_gemm_bf16_nn(const void *a, const void *b, void *c, int M, int N, int K, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -65,6 +65,8 @@ def lib() -> ctypes.CDLL:
         L.ave_attn_splitkv_workspace_bytes.restype = ctypes.c_size_t
         L.ave_gemm_bf16_tn.argtypes = [vp, vp, vp, ci, ci, ci, vp]
         L.ave_gemm_bf16_tn.restype = ci
+        L.ave_gemm_bf16_nn.argtypes = [vp, vp, vp, ci, ci, ci, vp]
+        L.ave_gemm_bf16_nn.restype = ci
         L.ave_attn_device_status.argtypes = [ctypes.POINTER(ctypes.c_uint)]
         L.ave_attn_device_status.restype = ci
         L.ave_attn_launch_count.argtypes = []
@@ -305,4 +307,29 @@ def ave_gemm_bf16_tn(a, b, c=None, stream=None):
                                     ctypes.c_void_p(c.data_ptr()), M, N, K, _stream_ptr(stream))
     if st != AVE_OK:
         raise AveAttnError(st, "ave_gemm_bf16_tn")
+    return c
+
+
+def ave_gemm_bf16_nn_raw(a_ptr, b_ptr, c_ptr, M, N, K, stream_ptr=None) -> int:
+    """The C call with plain integers for pointers; returns the status code."""
+    return int(lib().ave_gemm_bf16_nn(ctypes.c_void_p(a_ptr), ctypes.c_void_p(b_ptr), ctypes.c_void_p(c_ptr),
+                                      M, N, K, ctypes.c_void_p(stream_ptr)))
+
+
+def ave_gemm_bf16_nn(a, b, c=None, stream=None):
+    """C [M, N] = a [M, K] . b [K, N] on the tensors' CUDA device (contiguous bf16)."""
+    for t in (a, b):
+        if not (t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous() and t.dim() == 2):
+            raise ValueError("a and b must be contiguous 2-D CUDA bfloat16 tensors")
+    M, K = a.shape
+    Kb, N = b.shape
+    if Kb != K:
+        raise ValueError("a is [M, K] and b is [K, N]: the K sizes differ")
+    if c is None:
+        c = torch.empty((M, N), dtype=torch.bfloat16, device=a.device)
+    with torch.cuda.device(a.device):
+        st = lib().ave_gemm_bf16_nn(ctypes.c_void_p(a.data_ptr()), ctypes.c_void_p(b.data_ptr()),
+                                    ctypes.c_void_p(c.data_ptr()), M, N, K, _stream_ptr(stream))
+    if st != AVE_OK:
+        raise AveAttnError(st, "ave_gemm_bf16_nn")
     return c

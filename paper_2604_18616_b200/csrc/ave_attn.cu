@@ -308,15 +308,19 @@ int run_splitkv(const void *q, const void *k, const void *v, void *o, float *lse
 
 
 // C[M, N] = A[M, K] * B[N, K]^T: tensor maps of the three matrices, tile order, persistent launch.
-template <int TN>
-int launch_gemm_tn_tile(const void *a, const void *b, void *c, int M, int N, int K, int sms, cudaStream_t s) {
+template <int TN, bool B_NMAJOR>
+int launch_gemm_tile(const void *a, const void *b, void *c, int M, int N, int K, int sms, cudaStream_t s) {
     using Cfg = ave::GemmCfg<TN>;
     CUtensorMap ta, tb, tc;
     const Strides sa{(long long)M * K, (long long)M * K, (long long)K};
-    const Strides sb{(long long)N * K, (long long)N * K, (long long)K};
+    const Strides sb{(long long)N * K, (long long)N * K, (long long)(B_NMAJOR ? N : K)};
     const Strides sc{(long long)M * N, (long long)M * N, (long long)N};
     if (!encode_map(&ta, a, K, M, 1, 1, sa, Cfg::kTileM)) return AVE_ERR_CUDA;
-    if (!encode_map(&tb, b, K, N, 1, 1, sb, Cfg::kTileN)) return AVE_ERR_CUDA;
+    if (B_NMAJOR) {  // B [K, N]: rows of N elements, boxes of 64 columns x 64 rows of K
+        if (!encode_map(&tb, b, N, K, 1, 1, sb, Cfg::kSliceK)) return AVE_ERR_CUDA;
+    } else {         // B [N, K]: rows of K elements, boxes of 64 columns of K x the tile's rows
+        if (!encode_map(&tb, b, K, N, 1, 1, sb, Cfg::kTileN)) return AVE_ERR_CUDA;
+    }
     if (!encode_map(&tc, c, N, M, 1, 1, sc, Cfg::kOutBoxRows)) return AVE_ERR_CUDA;
     ave::GemmParams p;
     p.M = M;
@@ -327,7 +331,7 @@ int launch_gemm_tn_tile(const void *a, const void *b, void *c, int M, int N, int
     // The ~148 tiles in flight at a time should cover a near-square part of C, which minimises the A and B
     // bytes they pull through L2: 16 block rows x 9 block columns of 128 x 256 is 2048 x 2304 elements.
     p.group_m = 16;
-    auto kern = ave::gemm_bf16_tn_kernel<TN>;
+    auto kern = ave::gemm_bf16_kernel<TN, B_NMAJOR>;
     static std::atomic<bool> configured{false};  // per instantiation
     cudaError_t e;
     if (!configured.load(std::memory_order_acquire)) {
@@ -350,7 +354,8 @@ int launch_gemm_tn_tile(const void *a, const void *b, void *c, int M, int N, int
     return AVE_OK;
 }
 
-int launch_gemm_tn(const void *a, const void *b, void *c, int M, int N, int K, cudaStream_t s) {
+template <bool B_NMAJOR>
+int launch_gemm(const void *a, const void *b, void *c, int M, int N, int K, cudaStream_t s) {
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -362,8 +367,8 @@ int launch_gemm_tn(const void *a, const void *b, void *c, int M, int N, int K, c
     // finishes earlier (measured: n = 1024 gains a third, while at n = 2048, 128 tiles on 148 SMs, the narrow
     // tile's second wave costs a third)
     const long long wide_tiles = (long long)((M + 127) / 128) * ((N + 255) / 256);
-    if (2 * wide_tiles <= sms) return launch_gemm_tn_tile<128>(a, b, c, M, N, K, sms, s);
-    return launch_gemm_tn_tile<256>(a, b, c, M, N, K, sms, s);
+    if (2 * wide_tiles <= sms) return launch_gemm_tile<128, B_NMAJOR>(a, b, c, M, N, K, sms, s);
+    return launch_gemm_tile<256, B_NMAJOR>(a, b, c, M, N, K, sms, s);
 }
 
 }  // namespace
@@ -590,18 +595,32 @@ int ave_attn_trace_read(long long *out) {
 }
 #endif
 
-int ave_gemm_bf16_tn(const void *a, const void *b, void *c, int M, int N, int K, void *stream) {
+static int gemm_validate(const void *a, const void *b, const void *c, int M, int N, int K) {
     if (!a || !b || !c) return AVE_ERR_NULL_POINTER;
     if (M <= 0 || N <= 0 || K <= 0) return AVE_ERR_BAD_SHAPE;
     const long long lim = 1ll << 40;
     if ((long long)M * K >= lim || (long long)N * K >= lim || (long long)M * N >= lim) return AVE_ERR_BAD_SHAPE;
-    if ((long long)((M + 127) / 128) * ((N + 255) / 256) >= (1ll << 31)) return AVE_ERR_BAD_SHAPE;
+    if ((long long)((M + 127) / 128) * ((N + 127) / 128) >= (1ll << 31)) return AVE_ERR_BAD_SHAPE;
     if ((K & 7) || (N & 7)) return AVE_ERR_MISALIGNED;
     if ((reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b) | reinterpret_cast<uintptr_t>(c)) & 15u)
         return AVE_ERR_MISALIGNED;
-    int st = check_device();
+    return AVE_OK;
+}
+
+int ave_gemm_bf16_tn(const void *a, const void *b, void *c, int M, int N, int K, void *stream) {
+    int st = gemm_validate(a, b, c, M, N, K);
     if (st != AVE_OK) return st;
-    return launch_gemm_tn(a, b, c, M, N, K, static_cast<cudaStream_t>(stream));
+    st = check_device();
+    if (st != AVE_OK) return st;
+    return launch_gemm<false>(a, b, c, M, N, K, static_cast<cudaStream_t>(stream));
+}
+
+int ave_gemm_bf16_nn(const void *a, const void *b, void *c, int M, int N, int K, void *stream) {
+    int st = gemm_validate(a, b, c, M, N, K);
+    if (st != AVE_OK) return st;
+    st = check_device();
+    if (st != AVE_OK) return st;
+    return launch_gemm<true>(a, b, c, M, N, K, static_cast<cudaStream_t>(stream));
 }
 
 int ave_attn_last_cuda_error(void) { return t_last_cuda_error; }

@@ -1,5 +1,5 @@
-// Dense bf16 GEMM for sm_100a: C[M, N] = A[M, K] * B[N, K]^T, fp32 accumulation
-// in TMEM, bf16 result.  (The paper's first evaluated kernel family, Section 9:
+// Dense bf16 GEMM for sm_100a: C[M, N] = A[M, K] * B[N, K]^T (or A[M, K] * B[K, N]),
+// fp32 accumulation in TMEM, bf16 result.  (The paper's first evaluated kernel family, Section 9:
 // square bf16 matrices with normally distributed entries.)
 //
 // Persistent CTAs, one per SM, each walking output tiles of 128 x 256 (128 x 128
@@ -59,9 +59,12 @@ __device__ __forceinline__ void gemm_tile_coords(int id, const GemmParams &p, in
     bm = m0 + (rem - bn * gm);
 }
 
-template <int TN>
+// B_NMAJOR = false: B is [N, K] with K contiguous (C = A * B^T).  B_NMAJOR = true: B is [K, N] with N
+// contiguous (C = A * B); its slice then lands in shared memory as 64-column boxes of 64 K-rows each and is
+// read through an MN-major descriptor, so neither form needs a transposition.
+template <int TN, bool B_NMAJOR>
 __global__ void __launch_bounds__(256, 1)
-gemm_bf16_tn_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                     const __grid_constant__ CUtensorMap tm_c, const GemmParams p) {
     using Cfg = GemmCfg<TN>;
     constexpr int NS = Cfg::kStages;
@@ -133,7 +136,13 @@ gemm_bf16_tn_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                     const uint32_t dst = sRing + slot * Cfg::kStageBytes;
                     mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
                     tma_load_4d(dst, &tm_a, bar, ks * Cfg::kSliceK, bm * Cfg::kTileM, 0, 0);
-                    tma_load_4d(dst + Cfg::kABytes, &tm_b, bar, ks * Cfg::kSliceK, bn * Cfg::kTileN, 0, 0);
+                    if (!B_NMAJOR) {
+                        tma_load_4d(dst + Cfg::kABytes, &tm_b, bar, ks * Cfg::kSliceK, bn * Cfg::kTileN, 0, 0);
+                    } else {
+                        for (int x = 0; x < Cfg::kTileN / 64; ++x)  // boxes of 64 columns of B x 64 rows of K
+                            tma_load_4d(dst + Cfg::kABytes + x * (Cfg::kSliceK * 128), &tm_b, bar,
+                                        bn * Cfg::kTileN + x * 64, ks * Cfg::kSliceK, 0, 0);
+                    }
                 }
             }
         }
@@ -145,9 +154,15 @@ gemm_bf16_tn_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     } else if (warp == 1) {
         // =============================== MMA issuer ===============================
         const bool leader = elect_one();
-        constexpr uint32_t idesc = make_idesc_bf16(Cfg::kTileM, Cfg::kTileN, 0);
+        constexpr uint32_t idesc = make_idesc_bf16(Cfg::kTileM, Cfg::kTileN, B_NMAJOR ? 1 : 0);
         constexpr uint64_t desc_kmajor = make_sdesc_sw128(16, 1024);
         constexpr uint32_t hi = uint32_t(desc_kmajor >> 32), lo = uint32_t(desc_kmajor);
+        // N-contiguous B: 64-wide column groups are one box (64 K-rows x 128 B) apart, 8 K-rows 1024 B apart;
+        // 16 K-rows further is 16 x 128 B
+        constexpr uint64_t desc_nmajor = make_sdesc_sw128(Cfg::kSliceK * 128, 1024);
+        constexpr uint32_t hi_b = B_NMAJOR ? uint32_t(desc_nmajor >> 32) : hi;
+        constexpr uint32_t lo_b = B_NMAJOR ? uint32_t(desc_nmajor) : lo;
+        constexpr uint32_t b_kstep = B_NMAJOR ? ((16 * 128) >> 4) : (32 >> 4);
         bool ok = true;
         int ring = 0;
         int n_done = 0;  // tiles this CTA has issued so far
@@ -165,10 +180,10 @@ gemm_bf16_tn_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                 tc_fence_after();
                 if (leader) {
                     const uint32_t a_lo = lo | ((sRing + slot * Cfg::kStageBytes) >> 4);
-                    const uint32_t b_lo = lo | ((sRing + slot * Cfg::kStageBytes + Cfg::kABytes) >> 4);
+                    const uint32_t b_lo = lo_b | ((sRing + slot * Cfg::kStageBytes + Cfg::kABytes) >> 4);
 #pragma unroll
                     for (int kk = 0; kk < Cfg::kSliceK / 16; ++kk)
-                        umma_ss_words(d_tmem, a_lo + ((kk * 32) >> 4), hi, b_lo + ((kk * 32) >> 4), hi, idesc,
+                        umma_ss_words(d_tmem, a_lo + ((kk * 32) >> 4), hi, b_lo + kk * b_kstep, hi_b, idesc,
                                       (ks > 0 || kk > 0));
                     umma_commit(smem_u32(&bar_empty[slot]));
                     if (ks == n_slices - 1) umma_commit(smem_u32(&bar_acc_full[acc]));

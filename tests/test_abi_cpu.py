@@ -35,7 +35,7 @@ def test_header_declares_the_expected_entry_points():
     for n in ("ave_attn_fwd", "ave_attn_fwd_strided", "ave_attn_fwd_varlen", "ave_attn_fwd_host", "ave_attn_host_workspace_bytes", "ave_attn_device_status",
               "ave_attn_fwd_splitkv", "ave_attn_splitkv_workspace_bytes",
               "ave_attn_launch_count", "ave_attn_strerror", "ave_attn_version", "ave_attn_last_cuda_error",
-              "ave_gemm_bf16_tn"):
+              "ave_gemm_bf16_tn", "ave_gemm_bf16_nn"):
         assert n in names
 
 
@@ -119,3 +119,8 @@ def test_gemm_validation_before_any_cuda_call(lib):
     assert f(A, A, A, 128, 250, 64) == binding.AVE_ERR_MISALIGNED               # N not a multiple of 8
     assert f(A, A, A, 128, 256, 68) == binding.AVE_ERR_MISALIGNED               # K not a multiple of 8
     assert f(A + 8, A, A, 128, 256, 64) == binding.AVE_ERR_MISALIGNED
+    g = binding.ave_gemm_bf16_nn_raw
+    assert g(A, 0, A, 128, 256, 64) == binding.AVE_ERR_NULL_POINTER
+    assert g(A, A, A, 128, 0, 64) == binding.AVE_ERR_BAD_SHAPE
+    assert g(A, A, A, 128, 250, 64) == binding.AVE_ERR_MISALIGNED
+    assert g(A, A, A + 4, 128, 256, 64) == binding.AVE_ERR_MISALIGNED
