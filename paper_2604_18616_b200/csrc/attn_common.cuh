@@ -113,21 +113,4 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
     return false;
 }
 
-// The same with a non-suspending poll: the waiter notices the completion within a
-// few tens of cycles instead of after a wake-up, at the price of issue slots.
-// For the one warp whose reaction time is on the critical path.
-__device__ __forceinline__ bool mbar_spin_bounded(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                                  unsigned int code) {
-    for (uint32_t it = 0;; ++it) {
-        if (mbar_test_wait(bar, parity)) return true;
-        if ((it & 0x3FFu) == 0x3FFu) {
-            if (*abort_flag != 0) return false;
-            if (it >= (1u << 24)) break;  // 2^24 polls of a few tens of cycles each
-        }
-    }
-    *abort_flag = 1;
-    atomicOr(&g_device_status, code);
-    return false;
-}
-
 }  // namespace ave

@@ -307,10 +307,6 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const bool r = mbar_wait_bounded(smem_u32(bar), parity, &abort_flag, code);
         return __all_sync(0xffffffffu, r);
     };
-    auto spin_bar = [&](uint64_t *bar, uint32_t parity, unsigned code) -> bool {
-        const bool r = mbar_spin_bounded(smem_u32(bar), parity, &abort_flag, code);
-        return __all_sync(0xffffffffu, r);
-    };
     // Every consumer warp of the tile sequence calls this at the end of its n-th
     // tile to learn the next one (-1: none left); one lane releases the slot.
     auto next_tile = [&](int n, bool &ok) -> int {
@@ -524,7 +520,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     if (!ok) break;
                     const uint32_t v_addr = slot_addr(iv), k_addr = slot_addr(ik);
                     if (j < n0) {
-                        ok = spin_bar(&bar_p[0], np[0] & 1, STATUS_TIMEOUT_SOFTMAX);
+                        ok = wait_bar(&bar_p[0], np[0] & 1, STATUS_TIMEOUT_SOFTMAX);
                         if (!ok) break;
                         ++np[0];
                         if (n == kTraceTile && lane == 0) trace_stamp(0, j, 1);
@@ -540,7 +536,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         }
                     }
                     if (n == kTraceTile && lane == 0) trace_stamp(0, j, 2);
-                    ok = spin_bar(&bar_p[1], np[1] & 1, STATUS_TIMEOUT_SOFTMAX);
+                    ok = wait_bar(&bar_p[1], np[1] & 1, STATUS_TIMEOUT_SOFTMAX);
                     if (!ok) break;
                     ++np[1];
                     if (n == kTraceTile && lane == 0) trace_stamp(0, j, 3);
