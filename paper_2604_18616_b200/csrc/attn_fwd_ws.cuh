@@ -1,6 +1,8 @@
 // Attention forward, persistent warp-specialised kernel for sm_100a.
 //
-// A work tile is a block of 256 query rows of one (batch, head): two 128-row
+// A work tile is a block of 256 query rows of one (batch, head) - or, in causal
+// launches with an even number of query heads per key/value head, the same 128
+// query rows of two neighbouring heads: two 128-row
 // sub-tiles that ping-pong so the tensor pipe works on one while the softmax
 // of the other runs (the paper's "+Pipe": software pipelining across disjoint
 // groups of warps, Section 9; steps of the loop as in Section 2 / Fig. 1).
