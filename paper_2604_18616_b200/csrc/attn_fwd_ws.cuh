@@ -162,7 +162,7 @@ __device__ __forceinline__ TileOf<SPLIT, VARLEN> decode_tile(int id, const FwdPa
     // A unit is a (batch, head) pair or, when heads are paired, two neighbouring query heads of one
     // key/value head: the two sub-tiles then take the same 128 query rows of the two heads, so that in a
     // causal launch both visit the same key tiles and reach the diagonal, and the next tile, together.
-    const bool paired = !SPLIT && !VARLEN && p.pair_heads != 0;
+    const bool paired = !SPLIT && p.pair_heads != 0;
     const int per_group = p.heads_per_group * p.n_qblk;
     const int grp = id / per_group;
     const int rem = id - grp * per_group;
@@ -188,7 +188,7 @@ __device__ __forceinline__ TileOf<SPLIT, VARLEN> decode_tile(int id, const FwdPa
         w.sk = p.cu_k[w.b + 1] - w.k_base;
         // sub-tiles that start beyond the sequence's last query row have no rows and visit no keys
         w.n0 = (w.q0 < w.sq && w.sk > 0) ? kv_tiles_whole<CAUSAL>(w.q0, w.sq, w.sk) : 0;
-        w.n1 = (w.q0 + BM < w.sq && w.sk > 0) ? kv_tiles_whole<CAUSAL>(w.q0 + BM, w.sq, w.sk) : 0;
+        w.n1 = (w.q0 + w.dq < w.sq && w.sk > 0) ? kv_tiles_whole<CAUSAL>(w.q0 + w.dq, w.sq, w.sk) : 0;
         w.n1 = max(w.n0, w.n1);
     } else {
         w.n0 = kv_tiles_whole<CAUSAL>(w.q0, p.Sq, p.Sk);

@@ -194,7 +194,7 @@ int launch_attention(const void *q, const void *k, const void *v, void *o, float
     // Causal launches with an even number of query heads per key/value head give the two sub-tiles of a work
     // tile the same 128 query rows of two neighbouring heads instead of 256 rows of one head: both then visit
     // the same key tiles and finish together, where otherwise sub-tile 1 works through its diagonal step alone.
-    p.pair_heads = (causal && !split && !varlen && rows_per_head == 0 && G % 2 == 0) ? 1 : 0;
+    p.pair_heads = (causal && !split && rows_per_head == 0 && G % 2 == 0) ? 1 : 0;
     p.n_units = p.pair_heads ? p.BH / 2 : p.BH;
     const int rows_per_tile = p.pair_heads ? ave::BM : 2 * ave::BM;
     p.n_qblk = (Sq + rows_per_tile - 1) / rows_per_tile;
