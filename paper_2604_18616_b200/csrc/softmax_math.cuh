@@ -40,12 +40,15 @@ __device__ __forceinline__ float2 add2_round_down(float2 a, float2 b) {
 // taken from the mantissa of x + 1.5*2^23 (rounded down), 2^f from a cubic
 // fitted on [0, 1) (relative error < 9e-5, far below bf16 resolution), and
 // 2^n applied by adding n to the exponent field.  Inputs are clamped to
-// >= -126; inputs must stay below 2^22 - well above anything a probability
-// relative to a (possibly stale) row maximum can reach.
+// >= -127: there n = -127 and f = 0, the cubic gives exactly 1.0 and the
+// exponent field becomes 0, so every input <= -127, a masked score's -inf
+// included, yields exactly 0 (a row without visible keys must sum to 0).
+// Inputs must stay below 2^22 - well above anything a probability relative
+// to a (possibly stale) row maximum can reach.
 __device__ __forceinline__ float2 exp2_fma_pipe(float2 x) {
     const float kMagic = 12582912.f;  // 1.5 * 2^23
-    x.x = fmaxf(x.x, -126.f);
-    x.y = fmaxf(x.y, -126.f);
+    x.x = fmaxf(x.x, -127.f);
+    x.y = fmaxf(x.y, -127.f);
     const float2 t = add2_round_down(x, make_float2(kMagic, kMagic));
     const float2 n = __fadd2_rn(t, make_float2(-kMagic, -kMagic));
     const float2 f = __fadd2_rn(x, make_float2(-n.x, -n.y));
