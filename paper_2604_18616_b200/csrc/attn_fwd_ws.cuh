@@ -600,11 +600,6 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const int i0 = w.q0 + t * w.dq;
             const int i = i0 + r;                     // query row
             const int n_t = t ? w.n1 : w.n0;
-            // A warp whose 32 rows all lie beyond the last query row (few query rows against many keys,
-            // the ragged last block of a sequence) keeps up the barrier protocol but computes nothing:
-            // row r of O depends on row r of P only, so what the tensor pipe makes of those rows is
-            // never read.
-            const bool warp_active = i0 + wq * 32 < (SPLIT ? p.Sq : sq);
 
             if (n_t == 0) {
                 // no key visible to any row of this sub-tile: O = 0, LSE = -inf
@@ -646,12 +641,6 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     ++ns;
                     if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 1);
                     tc_fence_after();
-                    if (!warp_active) {
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(smem_u32(&bar_p[t]));
-                        return true;
-                    }
                     if (neg) {  // S_t <- -S_t in place (rare path, kept small)
 #pragma unroll 1
                         for (int c = 0; c < 8; ++c) {
@@ -804,11 +793,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     tc_fence_after();
                     const float inv_l = (l_run > 0.f) ? 1.f / l_run : 0.f;
                     const float lse_row = (l_run > 0.f) ? (m_run + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
-                    if (!warp_active) {  // nothing to store: hand O_t back
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(smem_u32(&bar_o_free[t]));
-                    } else if (SPLIT) {
+                    if (SPLIT) {
                         // partial result of this key range: normalised O in fp32 and its LSE, straight to global
                         const size_t row = (size_t(split_of(w)) * p.BH + bh) * p.Sq + i;
                         if (i < p.Sq) p.lse_partial[row] = lse_row;
