@@ -434,7 +434,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             // The whole warp runs this loop so that addresses and descriptors stay
             // warp-uniform; one elected lane issues the tcgen05 instructions.
             const bool leader = elect_one();
-            constexpr uint32_t idesc_qk = make_idesc_bf16(BM, BN, 0);
+            // A negative scale turns the row maximum of scale*s into the minimum of s; the softmax works
+            // with |scale| on scores the tensor pipe has negated (bit 13 of the descriptor negates A).
+            const uint32_t idesc_qk = make_idesc_bf16(BM, BN, 0) | ((p.scale_log2 < 0.f) ? (1u << 13) : 0u);
             constexpr uint32_t idesc_pv = make_idesc_bf16(BM, D, 1);
             constexpr uint64_t desc_kmajor = make_sdesc_sw128(16, 1024);
             constexpr uint64_t desc_v = make_sdesc_sw128(BN * 128, 1024);
@@ -577,11 +579,10 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const uint32_t tO = tmem + (t ? Cfg::kColO1 : Cfg::kColO0) + lane_sel;
         const uint32_t sO = sStage + t * Cfg::kStageOBytes + wq * (Cfg::kOutBoxRows * 128);  // this warp's 32 rows
         // The softmax works with a positive scale only, which keeps one maximum-then-exponentiate
-        // code path (the kernel's code has to stay within the instruction cache): a negative scale
-        // negates the scores in TMEM first and then uses |scale|; a zero scale (all visible keys
-        // weigh the same) is replaced by 2^-100, under which every visible score still rounds to
-        // an exponent of 0 while a masked one stays -inf.
-        const bool neg = p.scale_log2 < 0.f;
+        // code path (the kernel's code has to stay within the instruction cache): for a negative scale
+        // the MMA warp has the tensor pipe negate the scores and |scale| is used here; a zero scale
+        // (all visible keys weigh the same) is replaced by 2^-100, under which every visible score
+        // still rounds to an exponent of 0 while a masked one stays -inf.
         const float sl2 = (p.scale_log2 == 0.f) ? 7.888609052210118e-31f : fabsf(p.scale_log2);
         const bool tracer = (r == 0);
         uint32_t ns = 0;             // S_t tiles consumed so far (phase of bar_s[t])
@@ -641,18 +642,6 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     ++ns;
                     if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 1);
                     tc_fence_after();
-                    if (neg) {  // S_t <- -S_t in place (rare path, kept small)
-#pragma unroll 1
-                        for (int c = 0; c < 8; ++c) {
-                            uint32_t sc[16];
-                            tmem_ld_x16(tS + c * 16, sc);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int e = 0; e < 16; ++e) sc[e] ^= 0x80000000u;
-                            tmem_st_x16(tS + c * 16, sc);
-                        }
-                        tmem_wait_st();
-                    }
                     uint32_t sraw[4][32];
 #pragma unroll
                     for (int c = 0; c < 4; ++c) tmem_ld_x32(tS + c * 32, sraw[c]);
