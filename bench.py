@@ -31,8 +31,8 @@ DEFAULT_WORKLOAD = "c2_mha_prefill"
 NOMINAL_BF16_TFLOPS = 2250.0          # vendor dense bf16 figure, context only
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu captures summarised under
 # profiles/ (attn_fwd_ws_current_kernel_counters.md, gemm_bf16_tn_n8192_ncu_full.md); null for workloads that were not captured.
-NCU_DRAM_BYTES_PER_LAUNCH = {"c2_mha_prefill": 323.8e6, "c3_gqa_prefill": 266.2e6,
-                             "c4_long_context": 310.5e6, "c5_wide_noncausal": 563.9e6, "gemm_n8192": 1109.4e6}
+NCU_DRAM_BYTES_PER_LAUNCH = {"c2_mha_prefill": 323.7e6, "c3_gqa_prefill": 266.9e6,
+                             "c4_long_context": 311.4e6, "c5_wide_noncausal": 549.9e6, "gemm_n8192": 1109.4e6}
 FALLBACK_BF16_TFLOPS = 1590.0         # earlier measurement on this machine, used when no measured file exists
 
 
