@@ -22,6 +22,20 @@
  * reaches that point.  Inputs are never written; outputs must not alias inputs.
  * No call falls back to the CPU: without a compute-capability-10.0 device the
  * launch entry points return AVE_ERR_UNSUPPORTED_DEVICE or AVE_ERR_CUDA.
+ *
+ * Device-side time-outs are sticky.  Every wait inside a kernel is bounded; a
+ * wait that runs out records a code in a status word on that device, and from
+ * then on EVERY kernel of this library on that device (attention, split-KV,
+ * matrix product) returns at once without touching its outputs, while the
+ * launch entry points keep returning AVE_OK (they do not synchronise).  The
+ * condition ends when ave_attn_device_status() reads the word, which clears
+ * it.  A caller that wants to know whether its results are valid calls
+ * ave_attn_device_status() after the work of interest (it synchronises the
+ * device) and discards the outputs of every launch since the previous call if
+ * it reports AVE_ERR_DEVICE_TIMEOUT.
+ *
+ * A process may use several GPUs: every launch entry point prepares its kernel
+ * on the current device the first time it is used there.
  */
 #ifndef AVE_ATTN_H
 #define AVE_ATTN_H
@@ -43,7 +57,8 @@ typedef enum {
     AVE_ERR_CUDA = 7,               /* a CUDA call failed; see ave_attn_last_cuda_error() */
     AVE_ERR_DEVICE_TIMEOUT = 8,     /* a bounded wait inside a kernel gave up (ave_attn_device_status) */
     AVE_ERR_WORKSPACE = 9,          /* workspace NULL, misaligned or too small */
-    AVE_ERR_STATIC_SCRATCH = 10     /* the problem needs more scratch than the library's built-in array holds */
+    AVE_ERR_STATIC_SCRATCH = 10,    /* the problem needs more scratch than the library's built-in array holds */
+    AVE_ERR_KERNEL_IMAGE = 11       /* the compiled kernel cannot satisfy its own register split (miscompiled build) */
 } ave_status_t;
 
 /*
@@ -201,7 +216,11 @@ int ave_attn_fwd_splitkv_static(const void *q, const void *k, const void *v, voi
  * Synchronises the current device, then reads and clears the device-side
  * status word that kernels set when one of their bounded waits (on an
  * mbarrier) runs out.  Returns AVE_OK, AVE_ERR_DEVICE_TIMEOUT (with the raw
- * word in *raw_word if it is not NULL), or AVE_ERR_CUDA.
+ * word in *raw_word if it is not NULL), or AVE_ERR_CUDA.  Bits of the raw word:
+ * 1 a TMA load, 2 a tensor-core completion, 4 the softmax warps, 8 a ring slot
+ * or a tile-scheduler response did not arrive in time; 16 the wait of
+ * ave_attn_selftest_wait_timeout.  While the word is non-zero all kernels of the
+ * library on this device are no-ops (see "sticky" at the top of this file).
  */
 int ave_attn_device_status(unsigned int *raw_word);
 
@@ -216,6 +235,45 @@ int ave_attn_version(void);
 
 /* cudaError_t / CUresult of the last failing CUDA call on this thread. */
 int ave_attn_last_cuda_error(void);
+
+/*
+ * Diagnostics and self-tests.  (The paper has no counterpart to these; they
+ * exist so that the failure paths of the library can be exercised without
+ * faulting or hanging a GPU.)
+ *
+ * ave_attn_tensor_map_encodes: number of times the driver's tensor-map encoder
+ * has been called by this process.  The library keeps a small per-thread cache
+ * of encoded maps keyed by (pointer, shape, strides, box), so a repeated call
+ * on the same buffers encodes nothing.
+ *
+ * ave_attn_selftest_register_split: AVE_OK if a kernel image compiled with
+ * `regs_per_thread` registers per thread could satisfy the register split of
+ * the attention kernel's warp roles, else AVE_ERR_KERNEL_IMAGE.  The launch
+ * entry points apply the same test to the real image (cudaFuncGetAttributes)
+ * before a kernel's first launch on a device and refuse to launch on failure:
+ * a register request beyond the CTA's allocation would never return.  Host
+ * only; needs no GPU.
+ *
+ * ave_attn_selftest_inject_failures: make the next `count` kernel launches
+ * (what = AVE_INJECT_LAUNCH_FAILURE) or tensor-map encodes (what =
+ * AVE_INJECT_ENCODE_FAILURE) of this process fail on the host, before
+ * anything reaches the GPU: the affected entry point returns AVE_ERR_CUDA,
+ * ave_attn_last_cuda_error() holds the injected code, nothing is launched or
+ * counted, outputs are untouched.  count = 0 disarms.
+ *
+ * ave_attn_selftest_wait_timeout: enqueue a one-warp kernel whose only wait,
+ * on a barrier nobody arrives on, uses the library's bounded wait with a limit
+ * of 2^limit_cycles_log2 SM cycles (10..26).  The wait runs out, the kernel
+ * returns normally and bit 16 of the status word is set, after which the
+ * sticky no-op behaviour described at the top of this file can be observed and
+ * then cleared with ave_attn_device_status().
+ */
+#define AVE_INJECT_LAUNCH_FAILURE 1
+#define AVE_INJECT_ENCODE_FAILURE 2
+unsigned long long ave_attn_tensor_map_encodes(void);
+int ave_attn_selftest_register_split(int regs_per_thread);
+int ave_attn_selftest_inject_failures(int what, int count);
+int ave_attn_selftest_wait_timeout(int limit_cycles_log2, void *stream);
 
 #ifdef __cplusplus
 }

@@ -25,6 +25,10 @@ AVE_ERR_CUDA = 7
 AVE_ERR_DEVICE_TIMEOUT = 8
 AVE_ERR_WORKSPACE = 9
 AVE_ERR_STATIC_SCRATCH = 10
+AVE_ERR_KERNEL_IMAGE = 11
+INJECT_LAUNCH_FAILURE = 1
+INJECT_ENCODE_FAILURE = 2
+STATUS_BIT_SELFTEST = 16
 SPLITKV_STATIC_SCRATCH_BYTES = 8 << 20
 
 _lib = None
@@ -77,6 +81,14 @@ def lib() -> ctypes.CDLL:
         L.ave_attn_version.restype = ci
         L.ave_attn_last_cuda_error.argtypes = []
         L.ave_attn_last_cuda_error.restype = ci
+        L.ave_attn_tensor_map_encodes.argtypes = []
+        L.ave_attn_tensor_map_encodes.restype = ctypes.c_ulonglong
+        L.ave_attn_selftest_register_split.argtypes = [ci]
+        L.ave_attn_selftest_register_split.restype = ci
+        L.ave_attn_selftest_inject_failures.argtypes = [ci, ci]
+        L.ave_attn_selftest_inject_failures.restype = ci
+        L.ave_attn_selftest_wait_timeout.argtypes = [ci, vp]
+        L.ave_attn_selftest_wait_timeout.restype = ci
         _lib = L
     return _lib
 
@@ -97,8 +109,29 @@ def launch_count() -> int:
     return int(lib().ave_attn_launch_count())
 
 
+def tensor_map_encodes() -> int:
+    return int(lib().ave_attn_tensor_map_encodes())
+
+
+def selftest_register_split(regs_per_thread: int) -> int:
+    return int(lib().ave_attn_selftest_register_split(int(regs_per_thread)))
+
+
+def selftest_inject_failures(what: int, count: int) -> int:
+    return int(lib().ave_attn_selftest_inject_failures(int(what), int(count)))
+
+
+def selftest_wait_timeout(limit_cycles_log2: int = 16, stream=None) -> int:
+    return int(lib().ave_attn_selftest_wait_timeout(int(limit_cycles_log2), _stream_ptr(stream)))
+
+
 def device_status():
-    """(status, raw word) after synchronising the device."""
+    """(status, raw word) after synchronising the device; clears the word.
+
+    While the word is non-zero (a bounded wait inside a kernel ran out) every
+    kernel of the library on that device returns without writing its outputs,
+    although the launch calls keep returning AVE_OK: results since the previous
+    call of this function are valid only if it returns AVE_OK."""
     raw = ctypes.c_uint(0)
     st = lib().ave_attn_device_status(ctypes.byref(raw))
     return int(st), int(raw.value)

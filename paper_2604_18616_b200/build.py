@@ -2,10 +2,16 @@
 
 ``python -m paper_2604_18616_b200.build`` (or ``build_cuda()``) writes
 ``libave_attn.so`` next to this file.  nvcc cross-compiles without a GPU.
+
+The build reads ptxas' resource report and refuses an image in which an
+attention kernel got fewer registers per thread than its warp roles' register
+split draws on (``setmaxnreg.inc`` beyond the CTA's allocation never returns).
+The library repeats the check at run time on the loaded image.
 """
 from __future__ import annotations
 
 import os
+import re
 import subprocess
 import sys
 
@@ -18,12 +24,46 @@ NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",
     "-O3", "-std=c++17", "-lineinfo",
     "-shared", "-Xcompiler", "-fPIC",
+    "-Xptxas", "-v",
 ]
+
+# Register split of the attention kernel (WsCfg in csrc/attn_fwd_ws.cuh): 384 threads, of which one
+# warpgroup keeps 64 registers per thread and two take 216.
+ATTN_THREADS = 384
+ATTN_REGS_NEEDED = 128 * 64 + 256 * 216
 
 
 def _sources():
     return sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cuh"))) + \
-        [os.path.join(INCLUDE, "ave_attn.h")]
+        [os.path.join(INCLUDE, h) for h in sorted(os.listdir(INCLUDE)) if h.endswith(".h")]
+
+
+def kernel_registers(ptxas_report: str) -> dict:
+    """{mangled kernel name: registers per thread} from ``-Xptxas -v`` output."""
+    regs = {}
+    current = None
+    for line in ptxas_report.splitlines():
+        m = re.search(r"Compiling entry function '([^']+)'", line)
+        if m:
+            current = m.group(1)
+            continue
+        m = re.search(r"Used (\d+) registers", line)
+        if m and current:
+            regs[current] = int(m.group(1))
+            current = None
+    return regs
+
+
+def check_register_split(ptxas_report: str) -> dict:
+    """Raise if an attention kernel of the report cannot satisfy its register split."""
+    regs = {k: v for k, v in kernel_registers(ptxas_report).items() if "attn_fwd" in k}
+    if not regs:
+        raise RuntimeError("ptxas reported no attention kernel: cannot verify the register split")
+    for name, n in regs.items():
+        if ATTN_THREADS * n < ATTN_REGS_NEEDED:
+            raise RuntimeError("%s was compiled with %d registers per thread; its warp roles need %d x %d >= %d" % (
+                name, n, ATTN_THREADS, n, ATTN_REGS_NEEDED))
+    return regs
 
 
 def build_cuda(force: bool = False, verbose: bool = False) -> str:
@@ -32,9 +72,18 @@ def build_cuda(force: bool = False, verbose: bool = False) -> str:
         return LIB_PATH
     nvcc = os.environ.get("NVCC", "nvcc")
     tmp = LIB_PATH + ".tmp%d" % os.getpid()
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
-        ["-o", tmp, os.path.join(CSRC, "ave_attn.cu")]
-    subprocess.run(cmd, check=True)
+    cmd = [nvcc] + NVCC_FLAGS + ["-o", tmp, os.path.join(CSRC, "ave_attn.cu")]
+    r = subprocess.run(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
+    if verbose or r.returncode != 0:
+        sys.stderr.write(r.stdout)
+    if r.returncode != 0:
+        raise subprocess.CalledProcessError(r.returncode, cmd)
+    try:
+        check_register_split(r.stdout)
+    except Exception:
+        if os.path.exists(tmp):
+            os.remove(tmp)
+        raise
     os.replace(tmp, LIB_PATH)
     return LIB_PATH
 

@@ -7,11 +7,9 @@
 #include <cuda_runtime.h>
 
 #include "ptx_sm100.cuh"
+#include "work_tiles.cuh"
 
 namespace ave {
-
-constexpr int BM = 128;  // query rows per MMA tile (= TMEM lanes)
-constexpr int BN = 128;  // keys per step
 
 // Device-side status word; a kernel ORs a code in when a bounded wait gives up.
 // (This header is included by exactly one translation unit.)
@@ -21,40 +19,13 @@ constexpr unsigned int STATUS_TIMEOUT_LOAD = 1u;     // waiting for a TMA load
 constexpr unsigned int STATUS_TIMEOUT_MMA = 2u;      // waiting for a tcgen05.commit
 constexpr unsigned int STATUS_TIMEOUT_SOFTMAX = 4u;  // MMA warp waiting for P
 constexpr unsigned int STATUS_TIMEOUT_SLOT = 8u;     // producer waiting for a free stage
+constexpr unsigned int STATUS_TIMEOUT_SELFTEST = 16u; // the wait of the time-out self-test (meant to run out)
 
 // A wait is abandoned after this many SM clock cycles (a fraction of a second;
 // legitimate waits last microseconds).
 constexpr long long WAIT_LIMIT_CYCLES = 1ll << 29;
 // Poll limit of the short non-suspending drain loops that run after a wait was abandoned.
 constexpr uint32_t WAIT_LIMIT = 1u << 16;
-
-struct FwdParams {
-    void *o;          // bf16 [B, H, Sq, D] through the strides below
-    float *lse;       // fp32 [B, H, Sq]
-    long long o_stride_b, o_stride_h, o_stride_r;  // element strides of o (rows written without TMA use them)
-    int d_true;       // head dimension of the tensors (<= the kernel's D; TMA zero-fills / clips the rest)
-    int H, Hkv;       // query heads, key/value heads
-    int Sq, Sk;       // sequence lengths
-    int BH;           // B * H
-    int n_qblk;       // work tiles (blocks of 256 query rows) per (b, h)
-    int total_blocks; // grid size: n_qblk * n_units * n_splits
-    int pair_heads;   // != 0: a work tile is 128 query rows of two neighbouring query heads of one key/value head
-    int n_units;      // BH, or BH / 2 when heads are paired
-    int heads_per_group;  // units ((b, h) pairs, or pairs of heads) whose work tiles are launched together (their K/V share L2)
-    float scale_log2; // scale * log2(e)
-    int causal_off;   // key j is visible to query i iff j <= i + causal_off (Sk - Sq of the whole problem)
-    // Split-KV launches only: the keys are cut into n_splits ranges of keys_per_split (a multiple of
-    // BN); a work tile handles one range and writes a normalised fp32 partial result.
-    int n_splits;
-    int keys_per_split;
-    int rows_per_head;   // > 0: rows are (query head in group, query position) pairs, this many positions per head
-    // Variable-length launches only: sequence b owns query rows [cu_q[b], cu_q[b+1]) and key rows
-    // [cu_k[b], cu_k[b+1]) of token-major tensors [rows, heads, D]; Sq and Sk above are the maxima.
-    const int *cu_q, *cu_k;        // device, B + 1 entries each
-    long long lse_stride_h;        // lse is [H, total query rows]
-    float *o_partial;    // fp32 [n_splits, B*H, Sq, D]
-    float *lse_partial;  // fp32 [n_splits, B*H, Sq]
-};
 
 // tcgen05 instruction descriptor, kind::f16: fp32 accumulator, bf16 A and B,
 // A K-major (or in TMEM), B K-major (b_mn_major = 0) or MN-major (= 1).
@@ -78,9 +49,6 @@ __host__ __device__ constexpr uint64_t make_sdesc_sw128(uint32_t lbo_bytes, uint
            (1ull << 46)    // descriptor version for sm_100
            | (2ull << 61); // swizzle mode: 128 B
 }
-__device__ __forceinline__ uint64_t sdesc_at(uint64_t desc_no_addr, uint32_t smem_addr) {
-    return desc_no_addr | uint64_t((smem_addr >> 4) & 0x3FFFu);
-}
 
 // Optional role timeline (builds with -DAVE_TRACE=<cta index> only): SM clock
 // stamps of one CTA, [role][iteration][slot], read back by a debug entry point.
@@ -100,13 +68,13 @@ __device__ __forceinline__ void trace_stamp(int, int, int) {}
 // thread of the CTA has already given up; `abort_flag` is a shared-memory
 // word all roles watch.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                                  unsigned int code) {
+                                                  unsigned int code, long long limit_cycles = WAIT_LIMIT_CYCLES) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag != 0) return false;
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
+        if (clock64() - t0 > limit_cycles) break;
     }
     *abort_flag = 1;
     atomicOr(&g_device_status, code);

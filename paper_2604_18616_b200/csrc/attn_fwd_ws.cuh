@@ -82,148 +82,6 @@ __device__ __forceinline__ void setmaxnreg_dec() {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
 }
 
-// One work tile, decoded from its position in the launch order.
-struct WorkTileBase {
-    int bh;      // b * H + h
-    int b, h;    // batch and query head
-    int g;       // h / (H / Hkv): key/value head (Fig. 1: idx_h / gqa)
-    int q0;      // first query row
-    int dq, dh;  // sub-tile 1 relative to sub-tile 0: rows further down (BM, same head) or, in launches that
-                 // pair heads, the next query head of the same key/value head (same rows)
-    int n0, n1;  // key tiles the two sub-tiles visit (n1 >= n0)
-};
-template <bool SPLIT>
-struct WorkTileT : WorkTileBase {};
-template <>
-struct WorkTileT<true> : WorkTileBase {
-    int k_begin, k_end;  // keys [k_begin, k_end) belong to this tile (split-KV only; else the whole range)
-    int split;           // index of the key range
-};
-
-// Variable-length launches (never split): the tile also carries its sequence's lengths and first rows.
-struct WorkTileVar : WorkTileT<false> {
-    int sq, sk;          // this sequence's query and key counts
-    int q_base, k_base;  // its first row in the token-major Q/O and K/V tensors
-};
-template <bool SPLIT, bool VARLEN>
-using TileOf = std::conditional_t<VARLEN, WorkTileVar, WorkTileT<SPLIT>>;
-
-// Split-KV launches may pack the G query heads of a key/value head into the rows of one problem
-// ("head" = KV head, row r = head_in_group * rows_per_head + query position): the rows of Q, O and LSE
-// are contiguous that way, and only the causal mask needs the query position r % rows_per_head.
-// Smallest and one-past-largest query position among the rows [i0, i0 + BM):
-__device__ __forceinline__ int query_pos_lo(int i0, int rows_per_head) {
-    if (rows_per_head <= 0) return i0;
-    const int lo = i0 % rows_per_head;
-    return (lo + BM > rows_per_head) ? 0 : lo;
-}
-__device__ __forceinline__ int query_pos_hi(int i0, int rows_per_head) {
-    if (rows_per_head <= 0) return i0 + BM;
-    const int lo = i0 % rows_per_head;
-    return (lo + BM >= rows_per_head) ? rows_per_head : lo + BM;
-}
-
-// Number of key tiles a 128-row sub-tile must visit inside [k_begin, k_end); pos_hi is one past the
-// largest query position among its rows.
-template <bool CAUSAL>
-__device__ __forceinline__ int kv_tiles_for(int pos_hi, int causal_off, int k_begin, int k_end) {
-    int hi = k_end;
-    if (CAUSAL) hi = min(hi, pos_hi + causal_off);  // one past the last key any row of the sub-tile may see
-    return hi > k_begin ? (hi - k_begin + BN - 1) / BN : 0;
-}
-
-// The same count when the tile covers all keys [0, Sk): key j is visible to row i iff
-// j <= i + (Sk - Sq).
-template <bool CAUSAL>
-__device__ __forceinline__ int kv_tiles_whole(int i0, int Sq, int Sk) {
-    int n = (Sk + BN - 1) / BN;
-    if (CAUSAL) {
-        const int last_vis = i0 + BM - 1 + (Sk - Sq);  // last key the last row of the sub-tile may see
-        n = last_vis < 0 ? 0 : min(n, last_vis / BN + 1);
-    }
-    return n;
-}
-
-// Launch order: (batch, head) pairs in groups of p.heads_per_group (whose K/V
-// fit in L2 together); inside a group all heads' blocks of one query position,
-// longest (causal: last) position first.  Split-KV: the key ranges of one
-// (b, h, block) are adjacent in the order.
-template <bool CAUSAL, bool SPLIT, bool VARLEN = false>
-__device__ __forceinline__ TileOf<SPLIT, VARLEN> decode_tile(int id, const FwdParams &p) {
-    static_assert(!(SPLIT && VARLEN), "variable-length launches are not split");
-    TileOf<SPLIT, VARLEN> w;
-    int k_begin = 0, k_end = p.Sk;
-    if constexpr (SPLIT) {
-        w.split = id % p.n_splits;
-        id /= p.n_splits;
-        w.k_begin = k_begin = min(p.Sk, w.split * p.keys_per_split);
-        w.k_end = k_end = min(p.Sk, w.k_begin + p.keys_per_split);
-    }
-    // A unit is a (batch, head) pair or, when heads are paired, two neighbouring query heads of one
-    // key/value head: the two sub-tiles then take the same 128 query rows of the two heads, so that in a
-    // causal launch both visit the same key tiles and reach the diagonal, and the next tile, together.
-    const bool paired = !SPLIT && p.pair_heads != 0;
-    const int per_group = p.heads_per_group * p.n_qblk;
-    const int grp = id / per_group;
-    const int rem = id - grp * per_group;
-    const int u0 = grp * p.heads_per_group;
-    const int hg = min(p.heads_per_group, p.n_units - u0);
-    const int rank = rem / hg;
-    const int unit = u0 + (rem - rank * hg);
-    w.bh = paired ? 2 * unit : unit;
-    w.dq = paired ? 0 : BM;
-    w.dh = paired ? 1 : 0;
-    const int qb = CAUSAL ? (p.n_qblk - 1 - rank) : rank;
-    w.b = w.bh / p.H;
-    w.h = w.bh - w.b * p.H;
-    w.g = w.h / (p.H / p.Hkv);
-    w.q0 = qb * (paired ? BM : 2 * BM);
-    if constexpr (SPLIT) {
-        w.n0 = kv_tiles_for<CAUSAL>(query_pos_hi(w.q0, p.rows_per_head), p.causal_off, k_begin, k_end);
-        w.n1 = max(w.n0, kv_tiles_for<CAUSAL>(query_pos_hi(w.q0 + BM, p.rows_per_head), p.causal_off, k_begin, k_end));
-    } else if constexpr (VARLEN) {
-        w.q_base = p.cu_q[w.b];
-        w.k_base = p.cu_k[w.b];
-        w.sq = p.cu_q[w.b + 1] - w.q_base;
-        w.sk = p.cu_k[w.b + 1] - w.k_base;
-        // sub-tiles that start beyond the sequence's last query row have no rows and visit no keys
-        w.n0 = (w.q0 < w.sq && w.sk > 0) ? kv_tiles_whole<CAUSAL>(w.q0, w.sq, w.sk) : 0;
-        w.n1 = (w.q0 + w.dq < w.sq && w.sk > 0) ? kv_tiles_whole<CAUSAL>(w.q0 + w.dq, w.sq, w.sk) : 0;
-        w.n1 = max(w.n0, w.n1);
-    } else {
-        w.n0 = kv_tiles_whole<CAUSAL>(w.q0, p.Sq, p.Sk);
-        w.n1 = kv_tiles_whole<CAUSAL>(w.q0 + w.dq, p.Sq, p.Sk);
-    }
-    return w;
-}
-
-__device__ __forceinline__ int key_begin(const WorkTileT<false> &) { return 0; }
-__device__ __forceinline__ int key_begin(const WorkTileT<true> &w) { return w.k_begin; }
-__device__ __forceinline__ int key_end(const WorkTileT<false> &, const FwdParams &p) { return p.Sk; }
-__device__ __forceinline__ int key_end(const WorkTileT<true> &w, const FwdParams &) { return w.k_end; }
-__device__ __forceinline__ int split_of(const WorkTileT<false> &) { return 0; }
-__device__ __forceinline__ int split_of(const WorkTileT<true> &w) { return w.split; }
-__device__ __forceinline__ int key_end(const WorkTileVar &w, const FwdParams &) { return w.sk; }
-// Query/key counts and first rows of the tile's sequence; the tensor-map batch coordinate.
-template <class Tile> __device__ __forceinline__ int seq_q(const Tile &, const FwdParams &p) { return p.Sq; }
-template <class Tile> __device__ __forceinline__ int seq_k(const Tile &, const FwdParams &p) { return p.Sk; }
-template <class Tile> __device__ __forceinline__ int q_base_of(const Tile &) { return 0; }
-template <class Tile> __device__ __forceinline__ int k_base_of(const Tile &) { return 0; }
-template <class Tile> __device__ __forceinline__ int batch_coord(const Tile &w) { return w.b; }
-__device__ __forceinline__ int seq_q(const WorkTileVar &w, const FwdParams &) { return w.sq; }
-__device__ __forceinline__ int seq_k(const WorkTileVar &w, const FwdParams &) { return w.sk; }
-__device__ __forceinline__ int q_base_of(const WorkTileVar &w) { return w.q_base; }
-__device__ __forceinline__ int k_base_of(const WorkTileVar &w) { return w.k_base; }
-__device__ __forceinline__ int batch_coord(const WorkTileVar &) { return 0; }
-// Index of row i's log-sum-exp: [B, H, Sq], or [H, total rows] for variable-length launches.
-template <class Tile>
-__device__ __forceinline__ size_t lse_index(const Tile &w, const FwdParams &p, int i) {
-    return size_t(w.bh) * p.Sq + i;
-}
-__device__ __forceinline__ size_t lse_index(const WorkTileVar &w, const FwdParams &p, int i) {
-    return size_t(w.h) * p.lse_stride_h + w.q_base + i;
-}
-
 // ---- cluster launch control: take over the tile of a CTA that has not started
 __device__ __forceinline__ void clc_try_cancel(uint32_t response_smem, uint32_t bar) {
     asm volatile("clusterlaunchcontrol.try_cancel.async.shared::cta.mbarrier::complete_tx::bytes.b128 [%0], [%1];"
@@ -627,13 +485,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 // choice is made once per tile here: left as a run-time flag inside one body, the
                 // per-element compares and selects end up predicated into every step.
                 const int k_end = key_end(w, p);
-                int n_full = (k_end - key_begin(w)) / BN;
-                if (CAUSAL) {
-                    const int pos_lo = SPLIT ? query_pos_lo(i0, p.rows_per_head) : i0;
-                    const int num = pos_lo + off - key_begin(w) + 1;  // keys every row of the sub-tile sees
-                    n_full = min(n_full, num > 0 ? num / BN : 0);
-                }
-                n_full = max(0, min(n_full, n_t));
+                const int n_full = unmasked_steps<CAUSAL, SPLIT>(i0, n_t, key_begin(w), k_end, off, p.rows_per_head);
                 auto step = [&](const int j, auto masked_tag) -> bool {
                     constexpr bool need_mask = decltype(masked_tag)::value;
                     if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 0);

@@ -50,6 +50,16 @@ EncodeTiledFn encode_fn() {
     return f;
 }
 
+std::atomic<int> g_inject_launch_failures{0};  // test hook: the next launches fail before reaching the GPU
+std::atomic<int> g_inject_encode_failures{0};  // test hook: the next tensor-map encodes fail
+
+bool take_injected(std::atomic<int> &counter) {
+    int n = counter.load(std::memory_order_relaxed);
+    while (n > 0)
+        if (counter.compare_exchange_weak(n, n - 1, std::memory_order_relaxed)) return true;
+    return false;
+}
+
 // Element strides of one tensor's batch, head and row dimensions (the D elements of a row are contiguous).
 struct Strides {
     long long batch, head, row;
@@ -60,8 +70,45 @@ Strides contiguous_strides(int heads, int rows, int D) {
 
 // bf16 tensor [batch, heads, rows, D] with the given strides as a 4-D map {D, rows, heads, batch} with a
 // box of 64 columns x box_rows rows, 128-byte swizzle, zero fill outside the tensor.
+struct MapKey {
+    const void *base;
+    int D, rows, heads, batch, box_rows;
+    long long s_batch, s_head, s_row;
+    bool operator==(const MapKey &o) const {
+        return base == o.base && D == o.D && rows == o.rows && heads == o.heads && batch == o.batch &&
+               box_rows == o.box_rows && s_batch == o.s_batch && s_head == o.s_head && s_row == o.s_row;
+    }
+};
+// A tensor map is a pure function of its key (the encoder reads no device state), so repeated calls
+// on the same buffers, the common case in a serving loop, reuse the encoded 128 bytes.  Per thread,
+// direct-mapped, a few entries: no locks, and a collision only costs a re-encode.
+struct MapCache {
+    static constexpr int kEntries = 32;
+    MapKey key[kEntries];
+    CUtensorMap map[kEntries];
+    bool valid[kEntries] = {};
+    static unsigned slot_of(const MapKey &k) {
+        unsigned long long h = reinterpret_cast<uintptr_t>(k.base) * 0x9E3779B97F4A7C15ull;
+        h ^= (unsigned long long)(unsigned)k.rows * 0xC2B2AE3D27D4EB4Full + (unsigned)k.box_rows * 0x165667B19E3779F9ull +
+             (unsigned long long)k.s_row;
+        return unsigned(h >> 40) % kEntries;
+    }
+};
+thread_local MapCache t_map_cache;
+std::atomic<unsigned long long> g_map_encodes{0};  // encoder calls so far (a cache hit makes none)
+
 bool encode_map(CUtensorMap *map, const void *base, int D, int rows, int heads, int batch, const Strides &st,
                 int box_rows) {
+    if (take_injected(g_inject_encode_failures)) {
+        t_last_cuda_error = int(CUDA_ERROR_INVALID_VALUE);
+        return false;
+    }
+    const MapKey key{base, D, rows, heads, batch, box_rows, st.batch, st.head, st.row};
+    const unsigned slot = MapCache::slot_of(key);
+    if (t_map_cache.valid[slot] && t_map_cache.key[slot] == key) {
+        *map = t_map_cache.map[slot];
+        return true;
+    }
     EncodeTiledFn enc = encode_fn();
     if (!enc) return false;
     cuuint64_t gdim[4] = {cuuint64_t(D), cuuint64_t(rows), cuuint64_t(heads), cuuint64_t(batch)};
@@ -71,10 +118,14 @@ bool encode_map(CUtensorMap *map, const void *base, int D, int rows, int heads, 
     CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), gdim, gstride, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    g_map_encodes.fetch_add(1, std::memory_order_relaxed);
     if (r != CUDA_SUCCESS) {
         t_last_cuda_error = int(r);
         return false;
     }
+    t_map_cache.key[slot] = key;
+    t_map_cache.map[slot] = *map;
+    t_map_cache.valid[slot] = true;
     return true;
 }
 
@@ -121,19 +172,56 @@ int check_device() {
     return AVE_OK;
 }
 
+// Per kernel instantiation: the devices (by ordinal) on which the kernel has been prepared.  The
+// maximum dynamic shared-memory size is an attribute of a function ON ONE DEVICE, so a process that
+// drives several GPUs has to set it once per device, not once per process.
+struct PerDeviceOnce {
+    std::atomic<unsigned long long> done{0};
+    bool is_done(int dev) const { return dev >= 0 && dev < 64 && ((done.load(std::memory_order_acquire) >> dev) & 1ull); }
+    void mark(int dev) {
+        if (dev >= 0 && dev < 64) done.fetch_or(1ull << dev, std::memory_order_release);
+    }
+};
+
+// The softmax warps raise their register count with setmaxnreg.inc, which can only draw on what
+// the CTA was given at launch (threads x registers per thread as compiled).  A request beyond that
+// never returns, so a kernel image compiled with fewer registers than the split assumes must not
+// be launched at all.
+bool register_split_fits(int regs_per_thread_at_launch) {
+    using Cfg = ave::WsCfg<128>;
+    return 128 * Cfg::kRegsLight + 256 * Cfg::kRegsSoftmax <= Cfg::kThreads * regs_per_thread_at_launch;
+}
+
+template <class Kernel>
+int prepare_kernel(Kernel kern, int smem_bytes, bool check_register_split, PerDeviceOnce &once) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess && once.is_done(dev)) return AVE_OK;
+    if (e == cudaSuccess && check_register_split) {
+        cudaFuncAttributes attr;
+        e = cudaFuncGetAttributes(&attr, kern);
+        if (e == cudaSuccess && !register_split_fits(attr.numRegs)) return AVE_ERR_KERNEL_IMAGE;
+    }
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+    if (e != cudaSuccess) {
+        t_last_cuda_error = int(e);
+        return AVE_ERR_CUDA;
+    }
+    once.mark(dev);
+    return AVE_OK;
+}
+
 template <int D, bool CAUSAL, bool SPLIT, bool VARLEN = false>
 int launch_ws(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const CUtensorMap &to,
               const ave::FwdParams &p, cudaStream_t stream) {
     using Cfg = ave::WsCfg<D>;
     auto kern = ave::attn_fwd_ws_kernel<D, CAUSAL, SPLIT, VARLEN>;
-    static std::atomic<bool> configured{false};  // per instantiation
-    if (!configured.load(std::memory_order_acquire)) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
-        if (e != cudaSuccess) {
-            t_last_cuda_error = int(e);
-            return AVE_ERR_CUDA;
-        }
-        configured.store(true, std::memory_order_release);
+    static PerDeviceOnce once;  // per instantiation
+    const int st = prepare_kernel(kern, Cfg::kSmemBytes, true, once);
+    if (st != AVE_OK) return st;
+    if (take_injected(g_inject_launch_failures)) {
+        t_last_cuda_error = int(cudaErrorLaunchFailure);
+        return AVE_ERR_CUDA;
     }
     kern<<<dim3(p.total_blocks), dim3(Cfg::kThreads), Cfg::kSmemBytes, stream>>>(tq, tk, tv, to, p);
     cudaError_t e = cudaGetLastError();
@@ -174,7 +262,7 @@ int launch_attention(const void *q, const void *k, const void *v, void *o, float
     if (!encode_map(&tv, v, D, rows_k, Hkv, n_batch, sv, ave::BN)) return AVE_ERR_CUDA;
 
     const bool split = o_partial != nullptr;
-    ave::FwdParams p;
+    ave::FwdParams p{};
     p.o = o;
     p.lse = lse;
     p.o_stride_b = so.batch;
@@ -185,44 +273,10 @@ int launch_attention(const void *q, const void *k, const void *v, void *o, float
     p.cu_k = varlen ? varlen->cu_k : nullptr;
     p.lse_stride_h = varlen ? varlen->total_q : 0;
     const int Dk = D <= 64 ? 64 : 128;  // the kernel's head dimension: TMA zero-fills the columns beyond D
-    p.H = H;
-    p.Hkv = Hkv;
-    p.Sq = Sq;
-    p.Sk = Sk;
-    p.BH = B * H;
-    const int G = H / Hkv;
-    // Causal launches with an even number of query heads per key/value head give the two sub-tiles of a work
-    // tile the same 128 query rows of two neighbouring heads instead of 256 rows of one head: both then visit
-    // the same key tiles and finish together, where otherwise sub-tile 1 works through its diagonal step alone.
-    p.pair_heads = (causal && !split && rows_per_head == 0 && G % 2 == 0) ? 1 : 0;
-    p.n_units = p.pair_heads ? p.BH / 2 : p.BH;
-    const int rows_per_tile = p.pair_heads ? ave::BM : 2 * ave::BM;
-    p.n_qblk = (Sq + rows_per_tile - 1) / rows_per_tile;
-    p.causal_off = Sk - (rows_per_head > 0 ? rows_per_head : Sq);
-    p.rows_per_head = rows_per_head;
-    p.n_splits = split ? n_splits : 1;
-    p.keys_per_split = split ? keys_per_split : Sk;
+    if (!ave::plan_work_tiles(p, B, H, Hkv, Sq, Sk, D, causal != 0, split, n_splits, keys_per_split, rows_per_head))
+        return AVE_ERR_BAD_SHAPE;
     p.o_partial = o_partial;
     p.lse_partial = lse_partial;
-    const long long total = (long long)p.n_qblk * p.n_units * p.n_splits;
-    if (total >= (1ll << 31)) return AVE_ERR_BAD_SHAPE;
-    p.total_blocks = int(total);
-    {
-        // Launch units in groups whose K and V together stay within a slice of L2, whole key/value heads
-        // at a time: 32 MB, which keeps the re-reads of a group's K/V in L2 (measured on D = 64, long
-        // non-causal sequences: +3 % over 64 MB), unless that leaves a group with fewer than about three
-        // waves of work tiles on a 148-SM part (short sequences, many heads), where 64 MB measured better.
-        const long long kv_bytes_per_kv_head = 2ll * Sk * D * 2;
-        auto units_for = [&](long long budget) {
-            long long kv_heads = budget / kv_bytes_per_kv_head;
-            if (kv_heads < 1) kv_heads = 1;
-            long long upg = kv_heads * G / (p.pair_heads ? 2 : 1);
-            return upg > p.n_units ? (long long)p.n_units : upg;
-        };
-        long long upg = units_for(32ll << 20);
-        if (upg * p.n_qblk < 448) upg = units_for(64ll << 20);
-        p.heads_per_group = int(upg);
-    }
     p.scale_log2 = scale * 1.4426950408889634f;
 
     if (split) {
@@ -277,21 +331,26 @@ __global__ void splitkv_merge_kernel(const float *__restrict__ o_partial, const 
     if (ch == 0) lse[row] = (denom > 0.f) ? m + logf(denom) : -INFINITY;
 }
 
-// Keys per range: an equal share of Sk rounded up to whole key tiles.
-int splitkv_keys_per_split(int Sk, int n_splits) {
-    const long long share = ((long long)Sk + n_splits - 1) / n_splits;
-    return int((share + ave::BN - 1) / ave::BN * ave::BN);
+// One warp waits, with the library's bounded wait, on an mbarrier that nobody ever arrives on: the
+// wait must give up after `limit_cycles`, record its code in the device status word and return.
+__global__ void wait_timeout_selftest_kernel(long long limit_cycles) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        ave::mbar_init(ave::smem_u32(&bar), 1);
+        ave::fence_mbar_init();
+    }
+    __syncthreads();
+    ave::mbar_wait_bounded(ave::smem_u32(&bar), 0, &abort_flag, ave::STATUS_TIMEOUT_SELFTEST, limit_cycles);
 }
 
 int run_splitkv(const void *q, const void *k, const void *v, void *o, float *lse, int B, int H, int Hkv, int Sq,
                 int Sk, int D, int causal, float scale, int n_splits, float *o_partial, float *lse_partial,
                 cudaStream_t s) {
-    const int kps = splitkv_keys_per_split(Sk, n_splits);
-    // With grouped-query heads and few query rows, the G query heads of a KV head become rows of one
-    // problem with Hkv heads of G * Sq rows each: Q, O, LSE and the partials are laid out exactly the
-    // same in memory, and one work tile then serves up to 256 / Sq query heads per pass over K/V.
+    const int kps = ave::splitkv_keys_per_split(Sk, n_splits);
     const int G = H / Hkv;
-    const bool pack = G > 1 && Sq < 2 * ave::BM && (long long)G * Sq < (1ll << 30);
+    const bool pack = ave::splitkv_packs_heads(H, Hkv, Sq);  // query heads of a KV head as rows of one problem
     int st = pack ? launch_attention(q, k, v, o, lse, B, Hkv, Hkv, G * Sq, Sk, D, causal, scale, n_splits, kps,
                                      o_partial, lse_partial, Sq, nullptr, nullptr, s)
                   : launch_attention(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, causal, scale, n_splits, kps, o_partial,
@@ -337,16 +396,10 @@ int launch_gemm_tile(const void *a, const void *b, void *c, int M, int N, int K,
     // bytes they pull through L2: 16 block rows x 9 block columns of 128 x 256 is 2048 x 2304 elements.
     p.group_m = 16;
     auto kern = ave::gemm_bf16_kernel<TN, B_NMAJOR>;
-    static std::atomic<bool> configured{false};  // per instantiation
+    static PerDeviceOnce once;  // per instantiation
+    const int st = prepare_kernel(kern, Cfg::kSmemBytes, false, once);
+    if (st != AVE_OK) return st;
     cudaError_t e;
-    if (!configured.load(std::memory_order_acquire)) {
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
-        if (e != cudaSuccess) {
-            t_last_cuda_error = int(e);
-            return AVE_ERR_CUDA;
-        }
-        configured.store(true, std::memory_order_release);
-    }
     const long long n_tiles = (long long)p.tiles_m * p.tiles_n;
     const unsigned grid = unsigned(n_tiles < sms ? n_tiles : sms);
     kern<<<dim3(grid), dim3(Cfg::kThreads), Cfg::kSmemBytes, s>>>(ta, tb, tc, p);
@@ -584,11 +637,41 @@ const char *ave_attn_strerror(int status) {
         case AVE_ERR_WORKSPACE: return "workspace is NULL, misaligned or too small";
         case AVE_ERR_STATIC_SCRATCH:
             return "the problem needs more scratch than the built-in array of ave_attn_fwd_splitkv_static holds";
+        case AVE_ERR_KERNEL_IMAGE:
+            return "the compiled kernel has fewer registers per thread than its warp roles' register split needs";
         default: return "unknown status";
     }
 }
 
 int ave_attn_version(void) { return kVersion; }
+
+unsigned long long ave_attn_tensor_map_encodes(void) { return g_map_encodes.load(std::memory_order_relaxed); }
+
+int ave_attn_selftest_register_split(int regs_per_thread) {
+    return register_split_fits(regs_per_thread) ? AVE_OK : AVE_ERR_KERNEL_IMAGE;
+}
+
+int ave_attn_selftest_inject_failures(int what, int count) {
+    if (count < 0) return AVE_ERR_BAD_SHAPE;
+    if (what == AVE_INJECT_LAUNCH_FAILURE) g_inject_launch_failures.store(count, std::memory_order_relaxed);
+    else if (what == AVE_INJECT_ENCODE_FAILURE) g_inject_encode_failures.store(count, std::memory_order_relaxed);
+    else return AVE_ERR_BAD_SHAPE;
+    return AVE_OK;
+}
+
+int ave_attn_selftest_wait_timeout(int limit_cycles_log2, void *stream) {
+    if (limit_cycles_log2 < 10 || limit_cycles_log2 > 26) return AVE_ERR_BAD_SHAPE;  // 1 us .. a few tens of ms
+    int st = check_device();
+    if (st != AVE_OK) return st;
+    wait_timeout_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(1ll << limit_cycles_log2);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        t_last_cuda_error = int(e);
+        return AVE_ERR_CUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return AVE_OK;
+}
 
 #ifdef AVE_TRACE
 // Trace builds only (not part of the public interface): copies the role
@@ -603,7 +686,7 @@ int ave_attn_trace_read(long long *out) {
 static int gemm_validate(const void *a, const void *b, const void *c, int M, int N, int K) {
     if (!a || !b || !c) return AVE_ERR_NULL_POINTER;
     if (M <= 0 || N <= 0 || K <= 0) return AVE_ERR_BAD_SHAPE;
-    const long long lim = 1ll << 40;
+    const long long lim = 1ll << 39;  // elements: a tensor map holds byte strides below 2^40
     if ((long long)M * K >= lim || (long long)N * K >= lim || (long long)M * N >= lim) return AVE_ERR_BAD_SHAPE;
     if ((long long)((M + 127) / 128) * ((N + 127) / 128) >= (1ll << 31)) return AVE_ERR_BAD_SHAPE;
     if ((K & 7) || (N & 7)) return AVE_ERR_MISALIGNED;

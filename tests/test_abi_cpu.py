@@ -48,11 +48,11 @@ def test_library_exports_every_declared_symbol(lib):
 def test_version_and_strerror(lib):
     assert binding.version() >= 100
     seen = set()
-    for code in range(0, 10):
+    for code in range(0, 12):
         msg = binding.strerror(code)
         assert msg and msg != "unknown status"
         seen.add(msg)
-    assert len(seen) == 10
+    assert len(seen) == 12
     assert binding.strerror(12345) == "unknown status"
 
 
@@ -116,6 +116,7 @@ def test_gemm_validation_before_any_cuda_call(lib):
     assert f(A, A, A, 128, -8, 64) == binding.AVE_ERR_BAD_SHAPE
     assert f(A, A, A, 128, 256, 0) == binding.AVE_ERR_BAD_SHAPE
     assert f(A, A, A, 2 ** 21, 256, 2 ** 21) == binding.AVE_ERR_BAD_SHAPE      # M * K beyond 2^40
+    assert f(A, A, A, 2 ** 20, 256, 2 ** 19) == binding.AVE_ERR_BAD_SHAPE      # 2^39 elements: byte strides reach 2^40
     assert f(A, A, A, 128, 250, 64) == binding.AVE_ERR_MISALIGNED               # N not a multiple of 8
     assert f(A, A, A, 128, 256, 68) == binding.AVE_ERR_MISALIGNED               # K not a multiple of 8
     assert f(A + 8, A, A, 128, 256, 64) == binding.AVE_ERR_MISALIGNED
@@ -124,3 +125,41 @@ def test_gemm_validation_before_any_cuda_call(lib):
     assert g(A, A, A, 128, 0, 64) == binding.AVE_ERR_BAD_SHAPE
     assert g(A, A, A, 128, 250, 64) == binding.AVE_ERR_MISALIGNED
     assert g(A, A, A + 4, 128, 256, 64) == binding.AVE_ERR_MISALIGNED
+
+
+def test_register_split_guard(lib):
+    """The softmax warps' setmaxnreg.inc can only draw on threads x registers-at-launch; an image
+    compiled with fewer registers must be refused (128 x 64 + 256 x 216 = 63488 <= 384 x regs)."""
+    assert binding.selftest_register_split(168) == binding.AVE_OK
+    assert binding.selftest_register_split(166) == binding.AVE_OK
+    assert binding.selftest_register_split(165) == binding.AVE_ERR_KERNEL_IMAGE
+    assert binding.selftest_register_split(128) == binding.AVE_ERR_KERNEL_IMAGE
+    assert "register" in binding.strerror(binding.AVE_ERR_KERNEL_IMAGE)
+
+
+def test_build_checks_the_ptxas_register_report():
+    ok = ("ptxas info    : Compiling entry function '_ZN3ave18attn_fwd_ws_kernelILi128ELb1ELb0ELb0EEEvx' for 'sm_100a'\n"
+          "ptxas info    : Used 168 registers, used 1 barriers, 240 bytes smem\n"
+          "ptxas info    : Compiling entry function '_ZN3ave16gemm_bf16_kernelILi256ELb0EEEvx' for 'sm_100a'\n"
+          "ptxas info    : Used 94 registers, used 1 barriers\n")
+    regs = build.kernel_registers(ok)
+    assert sorted(regs.values()) == [94, 168]
+    assert list(build.check_register_split(ok).values()) == [168]       # the GEMM kernel has no register split
+    with pytest.raises(RuntimeError, match="registers per thread"):
+        build.check_register_split(ok.replace("Used 168", "Used 160"))
+    with pytest.raises(RuntimeError, match="no attention kernel"):
+        build.check_register_split("")
+    # the constants mirror the kernel's configuration
+    src = open(os.path.join(ROOT, "paper_2604_18616_b200", "csrc", "attn_fwd_ws.cuh")).read()
+    assert "kThreads = %d" % build.ATTN_THREADS in src
+    assert "kRegsLight = 64" in src and "kRegsSoftmax = 216" in src
+    assert build.ATTN_REGS_NEEDED == 128 * 64 + 256 * 216
+
+
+def test_selftest_hooks_validate_their_arguments(lib):
+    assert binding.selftest_inject_failures(3, 1) == binding.AVE_ERR_BAD_SHAPE
+    assert binding.selftest_inject_failures(binding.INJECT_LAUNCH_FAILURE, -1) == binding.AVE_ERR_BAD_SHAPE
+    assert binding.selftest_inject_failures(binding.INJECT_LAUNCH_FAILURE, 0) == binding.AVE_OK
+    assert binding.lib().ave_attn_selftest_wait_timeout(5, None) == binding.AVE_ERR_BAD_SHAPE
+    assert binding.lib().ave_attn_selftest_wait_timeout(40, None) == binding.AVE_ERR_BAD_SHAPE
+    assert binding.tensor_map_encodes() >= 0
