@@ -178,6 +178,14 @@ int ave_attn_fwd_splitkv(const void *q, const void *k, const void *v, void *o, f
 size_t ave_attn_splitkv_workspace_bytes(int B, int H, int Sq, int D, int n_splits);
 
 /*
+ * A reasonable n_splits for ave_attn_fwd_splitkv on the current device (148
+ * SMs assumed when there is none): enough key ranges that the work tiles fill
+ * the SMs several times over, no range shorter than 1024 keys, at most
+ * AVE_SPLITKV_MAX_SPLITS.  Host arithmetic only; 0 if an argument is invalid.
+ */
+int ave_attn_splitkv_default_splits(int B, int H, int Hkv, int Sq, int Sk, int D);
+
+/*
  * Split-KV attention for callers that must not allocate device memory.
  * (The paper has no counterpart to this entry point; it exists for deployment
  * reasons only.)

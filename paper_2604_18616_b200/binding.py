@@ -67,6 +67,8 @@ def lib() -> ctypes.CDLL:
         L.ave_attn_fwd_splitkv_static.restype = ci
         L.ave_attn_splitkv_workspace_bytes.argtypes = [ci] * 5
         L.ave_attn_splitkv_workspace_bytes.restype = ctypes.c_size_t
+        L.ave_attn_splitkv_default_splits.argtypes = [ci] * 6
+        L.ave_attn_splitkv_default_splits.restype = ci
         L.ave_gemm_bf16_tn.argtypes = [vp, vp, vp, ci, ci, ci, vp]
         L.ave_gemm_bf16_tn.restype = ci
         L.ave_gemm_bf16_nn.argtypes = [vp, vp, vp, ci, ci, ci, vp]
@@ -269,6 +271,10 @@ def ave_attn_fwd_host(q, k, v, o, lse, workspace, causal=False, scale=None, stre
 
 def splitkv_workspace_bytes(B, H, Sq, D, n_splits) -> int:
     return int(lib().ave_attn_splitkv_workspace_bytes(B, H, Sq, D, n_splits))
+
+
+def splitkv_default_splits(B, H, Hkv, Sq, Sk, D) -> int:
+    return int(lib().ave_attn_splitkv_default_splits(B, H, Hkv, Sq, Sk, D))
 
 
 def ave_attn_fwd_splitkv(q, k, v, n_splits, workspace=None, o=None, lse=None, causal=False, scale=None, stream=None):

@@ -544,6 +544,15 @@ size_t ave_attn_splitkv_workspace_bytes(int B, int H, int Sq, int D, int n_split
     return size_t(n_splits) * rows * (size_t(D) + 1) * sizeof(float);
 }
 
+int ave_attn_splitkv_default_splits(int B, int H, int Hkv, int Sq, int Sk, int D) {
+    if (B <= 0 || H <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0 || H % Hkv != 0 || (D != 64 && D != 128)) return 0;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        sms = 148;  // no device to ask: the count of the part this library is written for
+    return ave::splitkv_default_splits(B, H, Hkv, Sq, Sk, sms, AVE_SPLITKV_MAX_SPLITS);
+}
+
 int ave_attn_fwd_splitkv(const void *q, const void *k, const void *v, void *o, float *lse, int B, int H, int Hkv,
                          int Sq, int Sk, int D, int causal, float scale, int n_splits, void *workspace,
                          size_t workspace_bytes, void *stream) {

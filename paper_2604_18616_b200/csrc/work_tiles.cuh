@@ -265,4 +265,21 @@ inline bool splitkv_packs_heads(int H, int Hkv, int Sq) {
     return G > 1 && Sq < 2 * BM && (long long)G * Sq < (1ll << 30);
 }
 
+// A default number of key ranges for a split-KV launch on a part with `sms` SMs: enough ranges that the
+// work tiles fill the SMs several times over, but no range shorter than eight key tiles (shorter ranges
+// spend their time on the tile's fixed cost and on the merge).
+inline int splitkv_default_splits(int B, int H, int Hkv, int Sq, int Sk, int sms, int max_splits) {
+    const int G = H / Hkv;
+    const bool pack = splitkv_packs_heads(H, Hkv, Sq);
+    const long long rows = pack ? (long long)G * Sq : Sq;
+    const long long units = (long long)B * (pack ? Hkv : H) * ((rows + 2 * BM - 1) / (2 * BM));
+    const long long key_tiles = ((long long)Sk + BN - 1) / BN;
+    const long long target = 7ll * sms;  // about seven waves of work tiles
+    long long n = (target + units - 1) / units;
+    const long long longest = key_tiles / 8 > 0 ? key_tiles / 8 : 1;
+    if (n > longest) n = longest;
+    if (n > max_splits) n = max_splits;
+    return n < 1 ? 1 : int(n);
+}
+
 }  // namespace ave

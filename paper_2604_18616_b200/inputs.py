@@ -67,6 +67,16 @@ for _n in (1024, 2048, 4096, 8192, 16384):
         note="the paper's evaluation shape (LLaMA-3 70B prefill under 8-way TP)")
 
 
+# Decode: one new query token per sequence against a long key/value cache (the split-KV entry point);
+# bound by reading K and V once from HBM.
+for _name, _b, _h, _hkv, _sk, _seed in (("decode_mha_b8_k8192", 8, 32, 32, 8192, 201),
+                                        ("decode_gqa_b8_k16384", 8, 32, 8, 16384, 202),
+                                        ("decode_gqa_b1_k65536", 1, 32, 8, 65536, 203),
+                                        ("decode_gqa_b64_k4096", 64, 32, 8, 4096, 204)):
+    WORKLOADS[_name] = Workload(_name, _b, _h, _hkv, 1, _sk, 128, True, _seed,
+                                note="decode step: one query row per sequence, split-KV")
+
+
 def get(name: str) -> Workload:
     return WORKLOADS[name]
 

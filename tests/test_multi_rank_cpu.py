@@ -70,3 +70,26 @@ def test_two_ranks_gloo(tmp_path):
     out = tmp_path / "ok.txt"
     mp.spawn(_worker, args=(2, _free_port(), str(out)), nprocs=2, join=True)
     assert out.read_text() == "ok"
+
+
+@pytest.mark.parametrize("scaling", ["weak", "strong"])
+def test_bench_gpus_2_starts_two_ranks(scaling):
+    """`bench.py --gpus 2` with no torchrun environment starts the two ranks itself; `--plan-only` stops
+    after the rendezvous (gloo here, NCCL on GPUs) and reports which rank would run what."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--plan-only", "--scaling", scaling,
+                        "--workload", "c3_gqa_prefill"], capture_output=True, text=True, timeout=300, env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    line = json.loads([l for l in r.stdout.splitlines() if l.startswith("{")][-1])
+    assert line["n_gpus"] == 2 and line["scaling"] == scaling
+    plan = sorted(line["plan"], key=lambda p: p["rank"])
+    assert [p["rank"] for p in plan] == [0, 1] and [p["local_rank"] for p in plan] == [0, 1]
+    if scaling == "weak":          # an independent batch per rank
+        assert plan[0]["seed"] != plan[1]["seed"] and plan[0]["units"] == plan[1]["units"] == [0, 16]
+    else:                          # the (batch, KV head) units of one batch, split without overlap
+        assert plan[0]["seed"] == plan[1]["seed"]
+        assert plan[0]["units"] == [0, 8] and plan[1]["units"] == [8, 16]

@@ -1,5 +1,5 @@
 """The allocation-free split-KV entry point, checked against the workspace
-variant.
+variant and, like every other entry point, against the fp64 CPU oracle.
 
 ``ave_attn_fwd_splitkv_static`` is for callers that cannot give the library a
 workspace because they may not allocate device memory at the time of the call
@@ -15,6 +15,7 @@ import math
 import pytest
 import torch
 
+import oracle
 from paper_2604_18616_b200 import binding
 
 import parity
@@ -49,6 +50,10 @@ def both_entry_points(seed, B, H, Hkv, Sq, Sk, D, causal, n_splits):
     fin = torch.isfinite(lse_ref)
     assert torch.equal(torch.isfinite(lse), fin)
     assert (lse[fin] - lse_ref[fin]).abs().max().item() <= parity.LSE_TOL
+    # both entry points against the oracle on the same inputs
+    o_orc, lse_orc = oracle.attn_fwd(q.cpu(), k.cpu(), v.cpu(), causal, scale)
+    parity.compare(o_ref.cpu(), lse_ref.cpu(), o_orc, lse_orc, "workspace variant")
+    parity.compare(o.cpu(), lse.cpu(), o_orc, lse_orc, "built-in scratch variant")
 
 
 def test_two_calls_in_a_row_share_the_built_in_scratch():
