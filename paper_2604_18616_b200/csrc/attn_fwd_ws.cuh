@@ -67,11 +67,14 @@ constexpr float kRescaleThreshold = 8.0f;
 #endif
 constexpr unsigned kFmaPipeExpMask = AVE_FMA_EXP_MASK;
 
-// Trace builds record the role timeline of this one of a CTA's tiles (0 = its first).
+// Trace builds record the role timeline of two consecutive tiles of a CTA, starting at this one (0 = its first);
+// the second tile's steps follow at iteration index 32.
 #ifndef AVE_TRACE_TILE
 #define AVE_TRACE_TILE 0
 #endif
 constexpr int kTraceTile = AVE_TRACE_TILE;
+__device__ __forceinline__ bool traced(int n) { return unsigned(n - kTraceTile) < 2u; }
+__device__ __forceinline__ int trace_it(int n, int j) { return (n - kTraceTile) * 32 + (j < 30 ? j : 29); }
 
 template <int N>
 __device__ __forceinline__ void setmaxnreg_inc() {
@@ -117,7 +120,10 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     __shared__ __align__(16) unsigned long long clc_response[2][2];
     __shared__ __align__(8) uint64_t bar_q_full[2], bar_q_empty[2], bar_s[2], bar_p[2], bar_o[2], bar_o_free[2];
     __shared__ __align__(8) uint64_t bar_full[NS], bar_empty[NS];
-    __shared__ __align__(8) uint64_t bar_tile_full[2], bar_tile_empty[2], bar_drain;
+    __shared__ __align__(8) uint64_t bar_tile_full[2], bar_tile_ready[2], bar_tile_empty[2], bar_drain;
+    // The scheduler warp decodes every tile it obtains once, for all warps: index and decoded form, two in flight.
+    __shared__ int tile_id[2];
+    __shared__ TileOf<SPLIT, VARLEN> tile_info[2];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
@@ -143,6 +149,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             mbar_init(smem_u32(&bar_o[t]), 1);
             mbar_init(smem_u32(&bar_o_free[t]), 4);  // one arrival per softmax warp
             mbar_init(smem_u32(&bar_tile_full[t]), 1);
+            mbar_init(smem_u32(&bar_tile_ready[t]), 1);
             mbar_init(smem_u32(&bar_tile_empty[t]), Cfg::kTileConsumers);
         }
         mbar_init(smem_u32(&bar_drain), 1);
@@ -167,14 +174,14 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const bool r = mbar_wait_bounded(smem_u32(bar), parity, &abort_flag, code);
         return __all_sync(0xffffffffu, r);
     };
-    // Every consumer warp of the tile sequence calls this at the end of its n-th
-    // tile to learn the next one (-1: none left); one lane releases the slot.
-    auto next_tile = [&](int n, bool &ok) -> int {
+    // Every consumer warp of the tile sequence calls this to learn the tile after its n-th one (-1: none
+    // left) and takes the decoded tile from shared memory; one lane releases the slot.
+    auto next_tile = [&](int n, bool &ok, TileOf<SPLIT, VARLEN> &w_out) -> int {
         const int slot = n & 1;
-        ok = wait_bar(&bar_tile_full[slot], (n >> 1) & 1, STATUS_TIMEOUT_SLOT);
+        ok = wait_bar(&bar_tile_ready[slot], (n >> 1) & 1, STATUS_TIMEOUT_SLOT);
         if (!ok) return -1;
-        const int id = clc_decode(clc_response[slot]);
-        fence_proxy_async_smem();  // order the read before the slot's next asynchronous write
+        const int id = tile_id[slot];
+        if (id >= 0) w_out = tile_info[slot];
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bar_tile_empty[slot]));
         return id;
@@ -200,7 +207,16 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 }
                 ok = wait_bar(&bar_tile_full[slot], (k >> 1) & 1, STATUS_TIMEOUT_SLOT);
                 if (!ok) break;
-                if (clc_decode(clc_response[slot]) < 0) break;  // nothing left to take over: never ask again
+                const int id = clc_decode(clc_response[slot]);
+                fence_proxy_async_smem();  // order the read before the slot's next asynchronous write
+                if (id >= 0) {
+                    const TileOf<SPLIT, VARLEN> w = decode_tile<CAUSAL, SPLIT, VARLEN>(id, p);
+                    if (lane == 0) tile_info[slot] = w;
+                }
+                if (lane == 0) tile_id[slot] = id;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bar_tile_ready[slot]));
+                if (id < 0) break;  // nothing left to take over: never ask again
             }
         } else if (warp == 0) {
             // =============================== producer ===============================
@@ -213,43 +229,62 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             int ring = 0;  // K/V tiles loaded so far (ring position)
             bool ok = true;
             int id = blockIdx.x;
+            TileOf<SPLIT, VARLEN> w = decode_tile<CAUSAL, SPLIT, VARLEN>(id, p);
+            int q_tile[2] = {-1, -1};  // number of the tile whose Q_t was loaded last
             for (int n = 0; id >= 0 && ok; ++n) {
-                const TileOf<SPLIT, VARLEN> w = decode_tile<CAUSAL, SPLIT, VARLEN>(id, p);
-                // Q_t of this tile goes in as soon as the previous tile's last Q_t K^T has retired.
-                // Q_1 is released later than Q_0 (causal sub-tile 1 runs one step longer), and the
-                // first K/V tiles must not queue behind it, so a Q load that cannot go yet stays
-                // pending and is retried between the K/V loads.
-                bool q_pending[2] = {true, true};
-                auto try_load_q = [&](int t, bool blocking) {
-                    if (!q_pending[t]) return;
-                    if (n > 0) {
+                if (traced(n) && leader) trace_stamp(3, (n - kTraceTile) * 32 + 28, 0);
+                // The tile after this one, as soon as the scheduler warp has it: its Q_t can go in before this
+                // tile's last K and V do (Q comes from HBM, the K/V of a launch group mostly from L2).
+                int id_next = -2;  // -2: not known yet
+                TileOf<SPLIT, VARLEN> w_next = w;
+                // Q_t of tile number tn (this tile or the next) goes in as soon as the tile before it has issued
+                // its last Q_t K^T.  Q_1 is released later than Q_0 (causal sub-tile 1 runs one step longer), and
+                // the K/V tiles must not queue behind it, so a Q load that cannot go yet stays pending and is
+                // retried between the K/V loads.
+                auto try_load_q = [&](int t, int tn, const TileOf<SPLIT, VARLEN> &wt, bool blocking) {
+                    if (q_tile[t] != tn - 1) return;  // loaded already, or the tile before it is not in yet
+                    if (tn > 0) {
                         if (blocking) {
-                            ok = wait_bar(&bar_q_empty[t], (n - 1) & 1, STATUS_TIMEOUT_SLOT);
+                            ok = wait_bar(&bar_q_empty[t], (tn - 1) & 1, STATUS_TIMEOUT_SLOT);
                             if (!ok) return;
-                        } else if (!__all_sync(0xffffffffu, mbar_test_wait(smem_u32(&bar_q_empty[t]), (n - 1) & 1))) {
+                        } else if (!__all_sync(0xffffffffu, mbar_test_wait(smem_u32(&bar_q_empty[t]), (tn - 1) & 1))) {
                             return;
                         }
                     }
-                    q_pending[t] = false;
+                    q_tile[t] = tn;
                     if (leader) {
+                        if (traced(tn)) trace_stamp(3, (tn - kTraceTile) * 32 + 28, 1 + t);
                         const uint32_t bar = smem_u32(&bar_q_full[t]);
                         mbar_arrive_expect_tx(bar, Cfg::kTileBytes);
                         for (int x = 0; x < Cfg::kBoxes; ++x)  // the tensor maps are {D, rows, heads, batch}
                             tma_load_4d(sQ + t * Cfg::kTileBytes + x * Cfg::kBoxBytes, &tm_q, bar, x * 64,
-                                        q_base_of(w) + w.q0 + t * w.dq, w.h + t * w.dh, batch_coord(w));
+                                        q_base_of(wt) + wt.q0 + t * wt.dq, wt.h + t * wt.dh, batch_coord(wt));
                     }
                 };
-                try_load_q(0, false);
-                try_load_q(1, false);
+                bool near_end = w.n1 <= 2;  // the next tile is looked for only while this tile's last loads wait for their slots
+                auto poll_q = [&]() {
+                    try_load_q(0, n, w, false);
+                    try_load_q(1, n, w, false);
+                    if (!near_end) return;
+                    if (id_next == -2 &&
+                        __all_sync(0xffffffffu, mbar_test_wait(smem_u32(&bar_tile_ready[n & 1]), (n >> 1) & 1)))
+                        id_next = next_tile(n, ok, w_next);  // does not wait: the phase has completed
+                    if (id_next >= 0) {
+                        try_load_q(0, n + 1, w_next, false);
+                        try_load_q(1, n + 1, w_next, false);
+                    }
+                };
+                poll_q();
                 for (int it = 0; it < 2 * w.n1 && ok; ++it, ++ring) {  // it even: K_{it/2}; odd: V_{it/2}
                     const int slot = ring % NS, round = ring / NS;
+                    near_end = it + 4 >= 2 * w.n1;
                     if (round > 0) {
                         // Poll for the slot without blocking: a Q buffer may free up first, and the MMA
                         // warp may be waiting for that Q before it releases any more slots.
                         const long long t0 = clock64();
                         for (;;) {
-                            try_load_q(0, false);
-                            try_load_q(1, false);
+                            poll_q();
+                            if (!ok) break;
                             if (__all_sync(0xffffffffu, mbar_test_wait(smem_u32(&bar_empty[slot]), (round - 1) & 1))) break;
                             if (*reinterpret_cast<volatile int *>(&abort_flag) != 0) {
                                 ok = false;
@@ -265,22 +300,25 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         }
                         if (!ok) break;
                     } else {
-                        try_load_q(0, false);
-                        try_load_q(1, false);
+                        poll_q();
                     }
                     if (leader) {
                         const uint32_t bar = smem_u32(&bar_full[slot]);
                         const CUtensorMap *tm = (it & 1) ? &tm_v : &tm_k;
-                        if (n == kTraceTile) trace_stamp(3, it >> 1, it & 1);
+                        if (traced(n)) trace_stamp(3, trace_it(n, it >> 1), it & 1);
                         mbar_arrive_expect_tx(bar, Cfg::kTileBytes);
                         for (int x = 0; x < Cfg::kBoxes; ++x)
                             tma_load_4d(sRing + slot * Cfg::kTileBytes + x * Cfg::kBoxBytes, tm, bar, x * 64,
                                         k_base_of(w) + key_begin(w) + (it >> 1) * BN, w.g, batch_coord(w));
                     }
                 }
-                if (ok) try_load_q(0, true);
-                if (ok) try_load_q(1, true);
-                if (ok) id = next_tile(n, ok);
+                if (ok) try_load_q(0, n, w, true);
+                if (ok) try_load_q(1, n, w, true);
+                if (traced(n) && leader) trace_stamp(3, (n - kTraceTile) * 32 + 28, 3);
+                if (ok && id_next == -2) id_next = next_tile(n, ok, w_next);
+                if (traced(n) && leader) trace_stamp(3, (n - kTraceTile) * 32 + 28, 4);
+                id = id_next;
+                w = w_next;
             }
             if (!ok) {
                 // abandoned: give the loads still in flight a bounded chance to land
@@ -358,10 +396,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 const int n0 = w.n0, n1 = w.n1;
                 if (lane == 0) trace_stamp(3, n, 7);  // start of this CTA's n-th tile
                 // the tile after this one (its first steps are issued from inside this tile's loop)
-                const int id_next = next_tile(n, ok);
-                if (!ok) break;
                 TileOf<SPLIT, VARLEN> w_next = w;
-                if (id_next >= 0) w_next = decode_tile<CAUSAL, SPLIT, VARLEN>(id_next, p);
+                const int id_next = next_tile(n, ok, w_next);
+                if (!ok) break;
                 const int ring_next = ring + 2 * n1;
                 if (id_next >= 0 && n1 == 0) {  // nothing to do in this tile at all
                     start_subtile(0, w_next, n + 1, ring_next);
@@ -369,7 +406,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 }
                 for (int j = 0; j < n1 && ok; ++j) {
                     const int iv = ring + 2 * j + 1, ik = ring + 2 * j + 2;  // ring positions of V_j and K_{j+1}
-                    if (n == kTraceTile && lane == 0) trace_stamp(0, j, 0);
+                    if (traced(n) && lane == 0) trace_stamp(0, trace_it(n, j), 0);
                     // Everything this step needs from the ring and from the previous tile is checked
                     // first, while the softmax of this step is still running; after that only the two
                     // P hand-offs stand between this warp and the tensor pipe.
@@ -385,7 +422,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         ok = wait_bar(&bar_p[0], np[0] & 1, STATUS_TIMEOUT_SOFTMAX);
                         if (!ok) break;
                         ++np[0];
-                        if (n == kTraceTile && lane == 0) trace_stamp(0, j, 1);
+                        if (traced(n) && lane == 0) trace_stamp(0, trace_it(n, j), 1);
                         tc_fence_after();
                         issue_pv(0, v_addr, j == 0);
                         if (leader && j == n0 - 1) umma_commit(smem_u32(&bar_o[0]));
@@ -397,11 +434,11 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                             if (!ok) break;
                         }
                     }
-                    if (n == kTraceTile && lane == 0) trace_stamp(0, j, 2);
+                    if (traced(n) && lane == 0) trace_stamp(0, trace_it(n, j), 2);
                     ok = wait_bar(&bar_p[1], np[1] & 1, STATUS_TIMEOUT_SOFTMAX);
                     if (!ok) break;
                     ++np[1];
-                    if (n == kTraceTile && lane == 0) trace_stamp(0, j, 3);
+                    if (traced(n) && lane == 0) trace_stamp(0, trace_it(n, j), 3);
                     tc_fence_after();
                     issue_pv(1, v_addr, j == 0);
                     if (leader) umma_commit(smem_u32(&bar_empty[iv % NS]));
@@ -415,7 +452,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         if (ok) start_subtile(1, w_next, n + 1, ring_next);
                         if (!ok) break;
                     }
-                    if (n == kTraceTile && lane == 0) trace_stamp(0, j, 4);
+                    if (traced(n) && lane == 0) trace_stamp(0, trace_it(n, j), 4);
                 }
                 ring = ring_next;
                 id = id_next;
@@ -449,8 +486,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         bool store_pending = false;  // (lane 0) a TMA store may still be reading this warp's staging rows
 
         int id = blockIdx.x;
+        TileOf<SPLIT, VARLEN> w_tile = decode_tile<CAUSAL, SPLIT, VARLEN>(id, p);
         for (int n = 0; id >= 0 && ok; ++n) {
-            TileOf<SPLIT, VARLEN> w = decode_tile<CAUSAL, SPLIT, VARLEN>(id, p);
+            TileOf<SPLIT, VARLEN> w = w_tile;
             w.h += t * w.dh;                           // this sub-tile's query head (head-paired launches)
             w.bh += t * w.dh;
             const int bh = w.bh;
@@ -488,17 +526,17 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 const int n_full = unmasked_steps<CAUSAL, SPLIT>(i0, n_t, key_begin(w), k_end, off, p.rows_per_head);
                 auto step = [&](const int j, auto masked_tag) -> bool {
                     constexpr bool need_mask = decltype(masked_tag)::value;
-                    if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 0);
+                    if (traced(n) && tracer) trace_stamp(1 + t, trace_it(n, j), 0);
                     ok = wait_bar(&bar_s[t], ns & 1, STATUS_TIMEOUT_MMA);
                     if (!ok) return false;
                     ++ns;
-                    if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 1);
+                    if (traced(n) && tracer) trace_stamp(1 + t, trace_it(n, j), 1);
                     tc_fence_after();
                     uint32_t sraw[4][32];
 #pragma unroll
                     for (int c = 0; c < 4; ++c) tmem_ld_x32(tS + c * 32, sraw[c]);
                     tmem_wait_ld();
-                    if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 2);
+                    if (traced(n) && tracer) trace_stamp(1 + t, trace_it(n, j), 2);
 
                     const int j0 = key_begin(w) + j * BN;  // first key of this step
                     int lim = k_end - 1 - j0;           // columns c <= lim of this tile are visible to row i
@@ -606,17 +644,17 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                             }
                             if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) rescale_o(alpha);
                         }
-                        if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 3);
+                        if (traced(n) && tracer) trace_stamp(1 + t, trace_it(n, j), 3);
                         row_sum = exp_pass(m_run);
                     }
                     l_run = l_run * alpha + row_sum;
-                    if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 4);
+                    if (traced(n) && tracer) trace_stamp(1 + t, trace_it(n, j), 4);
 
                     tmem_wait_st();
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&bar_p[t]));
-                    if (n == kTraceTile && tracer) trace_stamp(1 + t, j, 5);
+                    if (traced(n) && tracer) trace_stamp(1 + t, trace_it(n, j), 5);
                     return true;
                 };
                 {
@@ -628,7 +666,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 }
 
                 // ---- epilogue: O / l -> bf16 -> shared (TMA layout) -> global; LSE = ln2 * (m + log2 l)
+                if (traced(n) && tracer) trace_stamp(1 + t, (n - kTraceTile) * 32 + 30, 0);
                 if (ok) ok = wait_bar(&bar_o[t], n_out & 1, STATUS_TIMEOUT_MMA);
+                if (traced(n) && tracer) trace_stamp(1 + t, (n - kTraceTile) * 32 + 30, 1);
                 if (ok) {
                     ++n_out;
                     tc_fence_after();
@@ -704,7 +744,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     }
                 }
             }
-            if (ok) id = next_tile(n, ok);
+            if (traced(n) && tracer) trace_stamp(1 + t, (n - kTraceTile) * 32 + 30, 2);
+            if (ok) id = next_tile(n, ok, w_tile);
+            if (traced(n) && tracer) trace_stamp(1 + t, (n - kTraceTile) * 32 + 30, 3);
         }
         if (lane == 0 && store_pending) tma_store_wait_all();
     }

@@ -80,18 +80,24 @@ struct MapKey {
     }
 };
 // A tensor map is a pure function of its key (the encoder reads no device state), so repeated calls
-// on the same buffers, the common case in a serving loop, reuse the encoded 128 bytes.  Per thread,
-// direct-mapped, a few entries: no locks, and a collision only costs a re-encode.
+// on the same buffers, the common case in a serving loop, reuse the encoded 128 bytes.  Per thread (no
+// locks), 16 entries searched linearly and replaced in turn: the handful of maps of one call always fit.
 struct MapCache {
-    static constexpr int kEntries = 32;
+    static constexpr int kEntries = 16;
     MapKey key[kEntries];
     CUtensorMap map[kEntries];
     bool valid[kEntries] = {};
-    static unsigned slot_of(const MapKey &k) {
-        unsigned long long h = reinterpret_cast<uintptr_t>(k.base) * 0x9E3779B97F4A7C15ull;
-        h ^= (unsigned long long)(unsigned)k.rows * 0xC2B2AE3D27D4EB4Full + (unsigned)k.box_rows * 0x165667B19E3779F9ull +
-             (unsigned long long)k.s_row;
-        return unsigned(h >> 40) % kEntries;
+    int next = 0;
+    const CUtensorMap *find(const MapKey &k) const {
+        for (int i = 0; i < kEntries; ++i)
+            if (valid[i] && key[i] == k) return &map[i];
+        return nullptr;
+    }
+    void insert(const MapKey &k, const CUtensorMap &m) {
+        key[next] = k;
+        map[next] = m;
+        valid[next] = true;
+        next = (next + 1) % kEntries;
     }
 };
 thread_local MapCache t_map_cache;
@@ -104,9 +110,8 @@ bool encode_map(CUtensorMap *map, const void *base, int D, int rows, int heads, 
         return false;
     }
     const MapKey key{base, D, rows, heads, batch, box_rows, st.batch, st.head, st.row};
-    const unsigned slot = MapCache::slot_of(key);
-    if (t_map_cache.valid[slot] && t_map_cache.key[slot] == key) {
-        *map = t_map_cache.map[slot];
+    if (const CUtensorMap *hit = t_map_cache.find(key)) {
+        *map = *hit;
         return true;
     }
     EncodeTiledFn enc = encode_fn();
@@ -123,9 +128,7 @@ bool encode_map(CUtensorMap *map, const void *base, int D, int rows, int heads, 
         t_last_cuda_error = int(r);
         return false;
     }
-    t_map_cache.key[slot] = key;
-    t_map_cache.map[slot] = *map;
-    t_map_cache.valid[slot] = true;
+    t_map_cache.insert(key, *map);
     return true;
 }
 

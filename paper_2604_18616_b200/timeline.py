@@ -1,0 +1,103 @@
+"""Role timeline of one CTA of the attention kernel (a profiling aid).
+
+``python -m paper_2604_18616_b200.timeline <workload> [--cta N] [--tile K]`` builds a trace variant
+of the library (``-DAVE_TRACE=<cta> -DAVE_TRACE_TILE=<k>``, written beside the normal one as
+``libave_attn_trace.so``), runs the named workload on cuda:0 and prints, in time order, the SM-clock
+stamps that the producer, MMA and softmax warps of that CTA took during its k-th and (k+1)-th work
+tiles: where a key step's time goes, and what a tile boundary costs.  The normal library carries no
+trace code.
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes
+import os
+import subprocess
+import sys
+
+from . import build
+
+TRACE_LIB = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libave_attn_trace.so")
+ROLES, ITERS, SLOTS = 4, 64, 8          # dimensions of the device-side stamp array
+NAMES = {0: "MMA", 1: "SM0", 2: "SM1", 3: "LD "}
+LABELS = {0: ["round start", "P0 taken", "PV0+QK0 issued", "P1 taken", "PV1+QK1 issued"],
+          1: ["wait S", "S ready", "S in registers", "row max done", "exp done", "P handed over"],
+          2: ["wait S", "S ready", "S in registers", "row max done", "exp done", "P handed over"],
+          3: ["K issue", "V issue"]}
+
+
+def build_trace_library(cta: int, tile: int) -> str:
+    nvcc = os.environ.get("NVCC", "nvcc")
+    flags = [f for f in build.NVCC_FLAGS if f not in ("-Xptxas", "-v")]
+    cmd = [nvcc] + flags + ["-DAVE_TRACE=%d" % cta, "-DAVE_TRACE_TILE=%d" % tile, "-o", TRACE_LIB,
+                            os.path.join(build.CSRC, "ave_attn.cu")]
+    subprocess.run(cmd, check=True)
+    return TRACE_LIB
+
+
+def events(stamps):
+    """[(clock, role name, text)] from the [ROLES][ITERS][SLOTS] stamp array (0 = not taken)."""
+    taken = [x for x in stamps if x > 0]
+    if not taken:
+        return []
+    base = min(taken)
+    out = []
+    for role in range(ROLES):
+        for it in range(ITERS):
+            for sl in range(SLOTS):
+                x = stamps[(role * ITERS + it) * SLOTS + sl]
+                if x <= 0:
+                    continue
+                tile, j = divmod(it, 32)
+                if role == 3 and sl == 7:
+                    text = "the CTA's tile number %d starts" % it
+                    who = "MMA"
+                elif j == 28:
+                    text = "T%d %s" % (tile, ["tile loop start", "Q0 issue", "Q1 issue", "all loads issued", "next tile known"][sl])
+                    who = NAMES[role]
+                elif j == 30:
+                    text = "T%d %s" % (tile, ["epilogue: wait for O", "epilogue: O ready", "epilogue done", "next tile known"][sl])
+                    who = NAMES[role]
+                else:
+                    lab = LABELS[role]
+                    text = "T%d j=%d %s" % (tile, j, lab[sl] if sl < len(lab) else "stamp %d" % sl)
+                    who = NAMES[role]
+                out.append((x - base, who, text))
+    out.sort()
+    return out
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser(description=__doc__.split("\n")[0])
+    ap.add_argument("workload")
+    ap.add_argument("--cta", type=int, default=0, help="blockIdx.x of the traced CTA")
+    ap.add_argument("--tile", type=int, default=0, help="first of the CTA's two traced tiles")
+    args = ap.parse_args(argv)
+    import torch
+    from . import binding, inputs
+    build_trace_library(args.cta, args.tile)
+    binding.LIB_PATH = TRACE_LIB
+    w = inputs.get(args.workload)
+    dev = torch.device("cuda:0")
+    q, k, v = [x.to(dev) for x in inputs.make_inputs(w)]
+    binding.ave_attn_fwd(q, k, v, causal=w.causal, scale=w.scale)     # one launch: stamps of several would mix
+    st, raw = binding.device_status()
+    if st != binding.AVE_OK:
+        raise RuntimeError("device status %d raw %#x" % (st, raw))
+    L = binding.lib()
+    buf = (ctypes.c_longlong * (ROLES * ITERS * SLOTS))()
+    L.ave_attn_trace_read.argtypes = [ctypes.c_void_p]
+    L.ave_attn_trace_read.restype = ctypes.c_int
+    if L.ave_attn_trace_read(buf) != 0:
+        raise RuntimeError("ave_attn_trace_read failed")
+    prev = {}
+    for x, who, text in events(list(buf)):
+        d = x - prev.get(who, x)
+        prev[who] = x
+        col = {"MMA": 0, "SM0": 1, "SM1": 2, "LD ": 3}[who]
+        print("%9d  %s%-4s +%-6d %s" % (x, " " * (26 * col), who, d, text))
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -55,3 +55,23 @@ def test_ceilings_of_the_narrow_head_kernel():
     # at D = 64 the exponential unit, not the tensor pipe, is the lower ceiling
     assert c["exp_unit_tflops"] < c["tensor_pipe_tflops"]
     assert 1100 < c["exp_unit_tflops"] < 1300 and 1800 < c["tensor_pipe_tflops"] < 2100
+
+
+def test_timeline_decodes_the_stamp_array():
+    """The profiling aid's host side: stamps [role][iteration][slot] -> time-ordered events; iterations 32.. belong
+    to the second traced tile, 28 / 30 are the producer's and the epilogue's per-tile stamps."""
+    from paper_2604_18616_b200 import timeline as t
+    st = [0] * (t.ROLES * t.ITERS * t.SLOTS)
+    at = lambda role, it, sl: (role * t.ITERS + it) * t.SLOTS + sl
+    st[at(3, 2, 7)] = 800
+    st[at(0, 3, 0)] = 900
+    st[at(1, 3, 1)] = 1000
+    st[at(2, 62, 2)] = 2000
+    st[at(3, 28, 1)] = 1500
+    ev = t.events(st)
+    assert [e[0] for e in ev] == [0, 100, 200, 700, 1200]
+    assert ev[0][1] == "MMA" and "tile number 2" in ev[0][2]
+    assert ev[2] == (200, "SM0", "T0 j=3 S ready")
+    assert ev[3] == (700, "LD ", "T0 Q0 issue")
+    assert ev[4] == (1200, "SM1", "T1 epilogue done")
+    assert t.events([0] * len(st)) == []
