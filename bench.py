@@ -75,6 +75,8 @@ def parse_args(argv=None):
     ap.add_argument("--sustain-seconds", type=float, default=1.5,
                     help="length of the extra back-to-back loop that shows the rate under the power cap (0: skip)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernel", type=int, default=0, choices=[0, 1, 2],
+                    help="attention kernel: 0 chosen per problem (default), 1 two sub-tiles per CTA, 2 one sub-tile per CTA")
     ap.add_argument("--plan-only", action="store_true",
                     help="start the ranks, print which rank runs what, and exit (gloo on a box without GPUs)")
     return ap.parse_args(argv)
@@ -338,6 +340,7 @@ class Ctx:
         if not torch.cuda.is_available():
             raise RuntimeError("bench.py needs a CUDA device: the attention path has no CPU fallback")
         binding.lib()   # raises if the CUDA library is not built
+        binding.select_kernel(self.args.kernel)
         torch.cuda.set_device(self.local_rank)
         self.dev = torch.device("cuda", self.local_rank)
         if self.world > 1:

@@ -179,9 +179,9 @@ size_t ave_attn_splitkv_workspace_bytes(int B, int H, int Sq, int D, int n_split
 
 /*
  * A reasonable n_splits for ave_attn_fwd_splitkv on the current device (148
- * SMs assumed when there is none): enough key ranges that the work tiles fill
- * the SMs several times over, no range shorter than 1024 keys, at most
- * AVE_SPLITKV_MAX_SPLITS.  Host arithmetic only; 0 if an argument is invalid.
+ * SMs assumed when there is none): the largest count with which all work
+ * tiles are resident at once (one wave), no range shorter than 256 keys, at
+ * most AVE_SPLITKV_MAX_SPLITS.  Host arithmetic only; 0 if an argument is invalid.
  */
 int ave_attn_splitkv_default_splits(int B, int H, int Hkv, int Sq, int Sk, int D);
 
@@ -231,6 +231,21 @@ int ave_attn_fwd_splitkv_static(const void *q, const void *k, const void *v, voi
  * library on this device are no-ops (see "sticky" at the top of this file).
  */
 int ave_attn_device_status(unsigned int *raw_word);
+
+/*
+ * The library has two attention kernels for the same operation: one whose CTAs
+ * process two 128-row sub-tiles of a 256-row work tile in lock-step (shared K/V
+ * loads; the default for long sequences and grouped-query heads), and one with
+ * a single 128-row sub-tile per CTA and two CTAs per SM (no lock-step at tile
+ * boundaries; better for short causal sequences).  which = 0 lets every call
+ * choose by problem shape (the default), 1 / 2 force the first / second for all
+ * later calls of this process.  Results agree within rounding order.  Returns
+ * AVE_OK, or AVE_ERR_BAD_SHAPE for another value.
+ */
+#define AVE_KERNEL_AUTO 0
+#define AVE_KERNEL_TWO_SUBTILES 1
+#define AVE_KERNEL_ONE_SUBTILE 2
+int ave_attn_select_kernel(int which);
 
 /* Number of kernels this library has launched in this process so far. */
 unsigned long long ave_attn_launch_count(void);

@@ -83,6 +83,8 @@ def lib() -> ctypes.CDLL:
         L.ave_attn_version.restype = ci
         L.ave_attn_last_cuda_error.argtypes = []
         L.ave_attn_last_cuda_error.restype = ci
+        L.ave_attn_select_kernel.argtypes = [ci]
+        L.ave_attn_select_kernel.restype = ci
         L.ave_attn_tensor_map_encodes.argtypes = []
         L.ave_attn_tensor_map_encodes.restype = ctypes.c_ulonglong
         L.ave_attn_selftest_register_split.argtypes = [ci]
@@ -109,6 +111,14 @@ def last_cuda_error() -> int:
 
 def launch_count() -> int:
     return int(lib().ave_attn_launch_count())
+
+
+KERNEL_AUTO, KERNEL_TWO_SUBTILES, KERNEL_ONE_SUBTILE = 0, 1, 2
+
+
+def select_kernel(which: int) -> int:
+    """0: choose per problem (default); 1: the two-sub-tile kernel; 2: the single-sub-tile kernel."""
+    return int(lib().ave_attn_select_kernel(int(which)))
 
 
 def tensor_map_encodes() -> int:

@@ -14,6 +14,7 @@
 #include <cuda_bf16.h>
 
 #include "attn_fwd_ws.cuh"
+#include "attn_fwd_1t.cuh"
 #include "gemm_bf16.cuh"
 
 // Scratch of ave_attn_fwd_splitkv_static: part of the device image, so every GPU that loads the
@@ -194,17 +195,31 @@ bool register_split_fits(int regs_per_thread_at_launch) {
     using Cfg = ave::WsCfg<128>;
     return 128 * Cfg::kRegsLight + 256 * Cfg::kRegsSoftmax <= Cfg::kThreads * regs_per_thread_at_launch;
 }
+bool register_split_fits_one_subtile(int regs_per_thread_at_launch) {
+    using Cfg = ave::OneCfg<128>;
+    return 128 * Cfg::kRegsLight + 128 * Cfg::kRegsSoftmax <= Cfg::kThreads * regs_per_thread_at_launch;
+}
 
+// Which attention kernel ordinary (not split-KV) launches use: 0 = chosen per problem, 1 = always the
+// two-sub-tile kernel, 2 = always the single-sub-tile kernel (ave_attn_select_kernel).
+std::atomic<int> g_kernel_choice{0};
+
+// check_register_split: 0 = none, 1 = the two-sub-tile kernel's split, 2 = the single-sub-tile kernel's
 template <class Kernel>
-int prepare_kernel(Kernel kern, int smem_bytes, bool check_register_split, PerDeviceOnce &once) {
+int prepare_kernel(Kernel kern, int smem_bytes, int check_register_split, PerDeviceOnce &once) {
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess && once.is_done(dev)) return AVE_OK;
     if (e == cudaSuccess && check_register_split) {
         cudaFuncAttributes attr;
         e = cudaFuncGetAttributes(&attr, kern);
-        if (e == cudaSuccess && !register_split_fits(attr.numRegs)) return AVE_ERR_KERNEL_IMAGE;
+        if (e == cudaSuccess && !(check_register_split == 1 ? register_split_fits(attr.numRegs)
+                                                            : register_split_fits_one_subtile(attr.numRegs)))
+            return AVE_ERR_KERNEL_IMAGE;
     }
+    // two CTAs of the single-sub-tile kernel share an SM: ask for the largest shared-memory carve-out
+    if (e == cudaSuccess && check_register_split == 2)
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) {
         t_last_cuda_error = int(e);
@@ -220,7 +235,7 @@ int launch_ws(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &t
     using Cfg = ave::WsCfg<D>;
     auto kern = ave::attn_fwd_ws_kernel<D, CAUSAL, SPLIT, VARLEN>;
     static PerDeviceOnce once;  // per instantiation
-    const int st = prepare_kernel(kern, Cfg::kSmemBytes, true, once);
+    const int st = prepare_kernel(kern, Cfg::kSmemBytes, 1, once);
     if (st != AVE_OK) return st;
     if (take_injected(g_inject_launch_failures)) {
         t_last_cuda_error = int(cudaErrorLaunchFailure);
@@ -236,6 +251,43 @@ int launch_ws(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &t
     return AVE_OK;
 }
 
+
+template <int D, bool CAUSAL, bool SPLIT, bool VARLEN = false>
+int launch_1t(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const ave::FwdParams &p,
+              cudaStream_t stream) {
+    using Cfg = ave::OneCfg<D>;
+    auto kern = ave::attn_fwd_1t_kernel<D, CAUSAL, SPLIT, VARLEN>;
+    static PerDeviceOnce once;  // per instantiation
+    const int st = prepare_kernel(kern, Cfg::kSmemBytes, 2, once);
+    if (st != AVE_OK) return st;
+    if (take_injected(g_inject_launch_failures)) {
+        t_last_cuda_error = int(cudaErrorLaunchFailure);
+        return AVE_ERR_CUDA;
+    }
+    kern<<<dim3(p.total_blocks), dim3(Cfg::kThreads), Cfg::kSmemBytes, stream>>>(tq, tk, tv, p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        t_last_cuda_error = int(e);
+        return AVE_ERR_CUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return AVE_OK;
+}
+
+// Whether an ordinary launch runs the single-sub-tile kernel (two CTAs per SM, 128-row tiles) instead of the
+// two-sub-tile one.
+bool use_one_subtile(int B, int H, int Hkv, int Sq, int Sk, int causal, bool split, bool varlen) {
+    const int choice = g_kernel_choice.load(std::memory_order_relaxed);
+    if (choice == 1) return false;
+    if (choice == 2) return true;
+    (void)B; (void)H; (void)Hkv; (void)Sk; (void)causal; (void)split; (void)varlen;
+    // At most 128 query rows per problem (decode, one chunk of a chunked prefill; Sq counts the packed rows of a
+    // head-packed split launch): the second sub-tile of a 256-row tile would be empty.  The single-sub-tile
+    // kernel then keeps two independent K/V streams per SM in flight, which is what an HBM-bound pass needs
+    // (measured on decode shapes: 0.63-0.66 -> 0.76-0.90 of the copy bandwidth).  With more rows the shared
+    // K/V loads of the two-sub-tile kernel win (measured 6-15 % on the prefill configurations).
+    return Sq <= ave::BM;
+}
 
 // Encode the tensor maps, fill the kernel parameters and launch.  n_splits == 1 with no partial
 // buffers is the ordinary forward; otherwise every work tile covers one range of keys_per_split keys
@@ -258,13 +310,14 @@ int launch_attention(const void *q, const void *k, const void *v, void *o, float
     const Strides sk = layout ? layout[1] : varlen ? token_major(Hkv, rows_k) : contiguous_strides(Hkv, Sk, D);
     const Strides sv = layout ? layout[2] : varlen ? token_major(Hkv, rows_k) : contiguous_strides(Hkv, Sk, D);
     const Strides so = layout ? layout[3] : varlen ? token_major(H, rows_q) : contiguous_strides(H, Sq, D);
+    const bool split = o_partial != nullptr;
+    const bool one = use_one_subtile(B, H, Hkv, Sq, Sk, causal, split, varlen != nullptr);
     CUtensorMap tq, tk, tv, to;
     if (!encode_map(&tq, q, D, rows_q, H, n_batch, sq, ave::BM)) return AVE_ERR_CUDA;
-    if (!encode_map(&to, o, D, rows_q, H, n_batch, so, ave::WsCfg<128>::kOutBoxRows)) return AVE_ERR_CUDA;
+    if (!one && !encode_map(&to, o, D, rows_q, H, n_batch, so, ave::WsCfg<128>::kOutBoxRows)) return AVE_ERR_CUDA;
     if (!encode_map(&tk, k, D, rows_k, Hkv, n_batch, sk, ave::BN)) return AVE_ERR_CUDA;
     if (!encode_map(&tv, v, D, rows_k, Hkv, n_batch, sv, ave::BN)) return AVE_ERR_CUDA;
 
-    const bool split = o_partial != nullptr;
     ave::FwdParams p{};
     p.o = o;
     p.lse = lse;
@@ -276,12 +329,29 @@ int launch_attention(const void *q, const void *k, const void *v, void *o, float
     p.cu_k = varlen ? varlen->cu_k : nullptr;
     p.lse_stride_h = varlen ? varlen->total_q : 0;
     const int Dk = D <= 64 ? 64 : 128;  // the kernel's head dimension: TMA zero-fills the columns beyond D
-    if (!ave::plan_work_tiles(p, B, H, Hkv, Sq, Sk, D, causal != 0, split, n_splits, keys_per_split, rows_per_head))
+    if (!ave::plan_work_tiles(p, B, H, Hkv, Sq, Sk, D, causal != 0, split, n_splits, keys_per_split, rows_per_head, one))
         return AVE_ERR_BAD_SHAPE;
     p.o_partial = o_partial;
     p.lse_partial = lse_partial;
     p.scale_log2 = scale * 1.4426950408889634f;
 
+    if (one) {
+        if (split) {
+            if (Dk == 128)
+                return causal ? launch_1t<128, true, true>(tq, tk, tv, p, s) : launch_1t<128, false, true>(tq, tk, tv, p, s);
+            return causal ? launch_1t<64, true, true>(tq, tk, tv, p, s) : launch_1t<64, false, true>(tq, tk, tv, p, s);
+        }
+        if (varlen) {
+            if (Dk == 128)
+                return causal ? launch_1t<128, true, false, true>(tq, tk, tv, p, s)
+                              : launch_1t<128, false, false, true>(tq, tk, tv, p, s);
+            return causal ? launch_1t<64, true, false, true>(tq, tk, tv, p, s)
+                          : launch_1t<64, false, false, true>(tq, tk, tv, p, s);
+        }
+        if (Dk == 128)
+            return causal ? launch_1t<128, true, false>(tq, tk, tv, p, s) : launch_1t<128, false, false>(tq, tk, tv, p, s);
+        return causal ? launch_1t<64, true, false>(tq, tk, tv, p, s) : launch_1t<64, false, false>(tq, tk, tv, p, s);
+    }
     if (split) {
         if (Dk == 128)
             return causal ? launch_ws<128, true, true>(tq, tk, tv, to, p, s) : launch_ws<128, false, true>(tq, tk, tv, to, p, s);
@@ -400,7 +470,7 @@ int launch_gemm_tile(const void *a, const void *b, void *c, int M, int N, int K,
     p.group_m = 16;
     auto kern = ave::gemm_bf16_kernel<TN, B_NMAJOR>;
     static PerDeviceOnce once;  // per instantiation
-    const int st = prepare_kernel(kern, Cfg::kSmemBytes, false, once);
+    const int st = prepare_kernel(kern, Cfg::kSmemBytes, 0, once);
     if (st != AVE_OK) return st;
     cudaError_t e;
     const long long n_tiles = (long long)p.tiles_m * p.tiles_n;
@@ -656,6 +726,12 @@ const char *ave_attn_strerror(int status) {
 }
 
 int ave_attn_version(void) { return kVersion; }
+
+int ave_attn_select_kernel(int which) {
+    if (which < 0 || which > 2) return AVE_ERR_BAD_SHAPE;
+    g_kernel_choice.store(which, std::memory_order_relaxed);
+    return AVE_OK;
+}
 
 unsigned long long ave_attn_tensor_map_encodes(void) { return g_map_encodes.load(std::memory_order_relaxed); }
 

@@ -34,6 +34,7 @@ struct FwdParams {
     int n_qblk;       // work tiles (blocks of query rows) per unit
     int total_blocks; // grid size: n_qblk * n_units * n_splits
     int pair_heads;   // != 0: a work tile is 128 query rows of two neighbouring query heads of one key/value head
+    int one_subtile;  // != 0: a work tile is 128 query rows of one head (the single-sub-tile kernel, two CTAs per SM)
     int n_units;      // BH, or BH / 2 when heads are paired
     int heads_per_group;  // units ((b, h) pairs, or pairs of heads) whose work tiles are launched together (their K/V share L2)
     float scale_log2; // scale * log2(e)
@@ -147,6 +148,7 @@ AVE_HD TileOf<SPLIT, VARLEN> decode_tile(int id, const FwdParams &p) {
     // key/value head: the two sub-tiles then take the same 128 query rows of the two heads, so that in a
     // causal launch both visit the same key tiles and reach the diagonal, and the next tile, together.
     const bool paired = !SPLIT && p.pair_heads != 0;
+    const bool single = p.one_subtile != 0;  // 128-row tiles with one sub-tile: dq = dh = 0 and n1 = n0
     const int per_group = p.heads_per_group * p.n_qblk;
     const int grp = id / per_group;
     const int rem = id - grp * per_group;
@@ -155,16 +157,16 @@ AVE_HD TileOf<SPLIT, VARLEN> decode_tile(int id, const FwdParams &p) {
     const int rank = rem / hg;
     const int unit = u0 + (rem - rank * hg);
     w.bh = paired ? 2 * unit : unit;
-    w.dq = paired ? 0 : BM;
+    w.dq = (paired || single) ? 0 : BM;
     w.dh = paired ? 1 : 0;
     const int qb = CAUSAL ? (p.n_qblk - 1 - rank) : rank;
     w.b = w.bh / p.H;
     w.h = w.bh - w.b * p.H;
     w.g = w.h / (p.H / p.Hkv);
-    w.q0 = qb * (paired ? BM : 2 * BM);
+    w.q0 = qb * ((paired || single) ? BM : 2 * BM);
     if constexpr (SPLIT) {
         w.n0 = kv_tiles_for<CAUSAL>(query_pos_hi(w.q0, p.rows_per_head), p.causal_off, k_begin, k_end);
-        w.n1 = imax(w.n0, kv_tiles_for<CAUSAL>(query_pos_hi(w.q0 + BM, p.rows_per_head), p.causal_off, k_begin, k_end));
+        w.n1 = single ? w.n0 : imax(w.n0, kv_tiles_for<CAUSAL>(query_pos_hi(w.q0 + BM, p.rows_per_head), p.causal_off, k_begin, k_end));
     } else if constexpr (VARLEN) {
         w.q_base = p.cu_q[w.b];
         w.k_base = p.cu_k[w.b];
@@ -173,7 +175,7 @@ AVE_HD TileOf<SPLIT, VARLEN> decode_tile(int id, const FwdParams &p) {
         // sub-tiles that start beyond the sequence's last query row have no rows and visit no keys
         w.n0 = (w.q0 < w.sq && w.sk > 0) ? kv_tiles_whole<CAUSAL>(w.q0, w.sq, w.sk) : 0;
         w.n1 = (w.q0 + w.dq < w.sq && w.sk > 0) ? kv_tiles_whole<CAUSAL>(w.q0 + w.dq, w.sq, w.sk) : 0;
-        w.n1 = imax(w.n0, w.n1);
+        w.n1 = imax(w.n0, w.n1);  // (one sub-tile: dq = 0, so n1 = n0)
     } else {
         w.n0 = kv_tiles_whole<CAUSAL>(w.q0, p.Sq, p.Sk);
         w.n1 = kv_tiles_whole<CAUSAL>(w.q0 + w.dq, p.Sq, p.Sk);
@@ -213,7 +215,7 @@ AVE_HD size_t lse_index(const WorkTileVar &w, const FwdParams &p, int i) {
 // split launch whose rows pack the query heads of a key/value head (H == Hkv there).  Returns false
 // when the grid would not fit in 31 bits.
 inline bool plan_work_tiles(FwdParams &p, int B, int H, int Hkv, int Sq, int Sk, int D, bool causal, bool split,
-                            int n_splits, int keys_per_split, int rows_per_head) {
+                            int n_splits, int keys_per_split, int rows_per_head, bool one_subtile = false) {
     p.H = H;
     p.Hkv = Hkv;
     p.Sq = Sq;
@@ -223,9 +225,10 @@ inline bool plan_work_tiles(FwdParams &p, int B, int H, int Hkv, int Sq, int Sk,
     // Causal launches with an even number of query heads per key/value head give the two sub-tiles of a work
     // tile the same 128 query rows of two neighbouring heads instead of 256 rows of one head: both then visit
     // the same key tiles and finish together, where otherwise sub-tile 1 works through its diagonal step alone.
-    p.pair_heads = (causal && !split && rows_per_head == 0 && G % 2 == 0) ? 1 : 0;
+    p.one_subtile = one_subtile ? 1 : 0;
+    p.pair_heads = (causal && !split && rows_per_head == 0 && G % 2 == 0 && !one_subtile) ? 1 : 0;
     p.n_units = p.pair_heads ? p.BH / 2 : p.BH;
-    const int rows_per_tile = p.pair_heads ? BM : 2 * BM;
+    const int rows_per_tile = (p.pair_heads || one_subtile) ? BM : 2 * BM;
     p.n_qblk = (Sq + rows_per_tile - 1) / rows_per_tile;
     p.causal_off = Sk - (rows_per_head > 0 ? rows_per_head : Sq);
     p.rows_per_head = rows_per_head;
@@ -265,19 +268,22 @@ inline bool splitkv_packs_heads(int H, int Hkv, int Sq) {
     return G > 1 && Sq < 2 * BM && (long long)G * Sq < (1ll << 30);
 }
 
-// A default number of key ranges for a split-KV launch on a part with `sms` SMs: enough ranges that the
-// work tiles fill the SMs several times over, but no range shorter than eight key tiles (shorter ranges
-// spend their time on the tile's fixed cost and on the merge).
+// A default number of key ranges for a split-KV launch on a part with `sms` SMs: the largest count with
+// which all work tiles are still resident at once (one CTA per SM for 256-row tiles, two for problems of at
+// most 128 rows, which run the single-sub-tile kernel), so that the whole launch is one wave; measured on
+// decode shapes, a second, partial wave costs more than longer key ranges do.  No range shorter than two
+// key tiles.
 inline int splitkv_default_splits(int B, int H, int Hkv, int Sq, int Sk, int sms, int max_splits) {
     const int G = H / Hkv;
     const bool pack = splitkv_packs_heads(H, Hkv, Sq);
     const long long rows = pack ? (long long)G * Sq : Sq;
-    const long long units = (long long)B * (pack ? Hkv : H) * ((rows + 2 * BM - 1) / (2 * BM));
+    const bool one = rows <= BM;
+    const long long rows_per_tile = one ? BM : 2 * BM;
+    const long long units = (long long)B * (pack ? Hkv : H) * ((rows + rows_per_tile - 1) / rows_per_tile);
+    const long long resident = one ? 2ll * sms : sms;
     const long long key_tiles = ((long long)Sk + BN - 1) / BN;
-    const long long target = 7ll * sms;  // about seven waves of work tiles
-    long long n = (target + units - 1) / units;
-    const long long longest = key_tiles / 8 > 0 ? key_tiles / 8 : 1;
-    if (n > longest) n = longest;
+    long long n = resident / units;
+    if (n > key_tiles / 2) n = key_tiles / 2;
     if (n > max_splits) n = max_splits;
     return n < 1 ? 1 : int(n);
 }

@@ -67,8 +67,12 @@ def visible(sq, sk, causal):
     return (j <= i + (sk - sq)) if causal else np.ones((sq, sk), dtype=bool)
 
 
-def check_launch(wt, B, H, Hkv, Sq, Sk, D, causal, n_splits=0, cu_q=None, cu_k=None):
-    plan, tiles = decode(wt, B, H, Hkv, Sq, Sk, D, causal, n_splits, cu_q, cu_k)
+def check_launch(wt, B, H, Hkv, Sq, Sk, D, causal, n_splits=0, cu_q=None, cu_k=None, one=False):
+    wt.wt_set_one_subtile(int(one))
+    try:
+        plan, tiles = decode(wt, B, H, Hkv, Sq, Sk, D, causal, n_splits, cu_q, cu_k)
+    finally:
+        wt.wt_set_one_subtile(0)
     varlen = cu_q is not None
     G = H // Hkv
     ns = max(1, n_splits)
@@ -76,6 +80,8 @@ def check_launch(wt, B, H, Hkv, Sq, Sk, D, causal, n_splits=0, cu_q=None, cu_k=N
     if n_splits:
         assert plan.keys_per_split % BN == 0 and plan.keys_per_split * n_splits >= Sk
         assert plan.packed == int(G > 1 and Sq < 2 * BM)
+    elif one:
+        assert plan.pair_heads == 0 and plan.n_qblk == -(-Sq // BM)
     else:
         assert plan.pair_heads == int(bool(causal) and G % 2 == 0)
     seq = [(cu_q[b + 1] - cu_q[b], cu_k[b + 1] - cu_k[b]) for b in range(B)] if varlen else [(Sq, Sk)] * B
@@ -93,7 +99,9 @@ def check_launch(wt, B, H, Hkv, Sq, Sk, D, causal, n_splits=0, cu_q=None, cu_k=N
         assert w.n0 <= w.n1
         vis = masks[(sq, sk)]
         needed0 = None
-        for t in (0, 1):
+        if one:  # 128-row tiles: the kernel has a single sub-tile and reads n0 only
+            assert (w.dq, w.dh) == (0, 0) and w.n1 == w.n0
+        for t in ((0,) if one else (0, 1)):
             head = w.h + t * w.dh
             i0 = w.q0 + t * w.dq
             n_t, n_full = (w.n1, w.n_full1) if t else (w.n0, w.n_full0)
@@ -181,6 +189,16 @@ def test_split_kv_launches_with_and_without_packed_heads(wt, B, H, Hkv, Sq, Sk, 
     check_launch(wt, B, H, Hkv, Sq, Sk, D, causal, n_splits=n_splits)
 
 
+@pytest.mark.parametrize("B,H,Hkv,Sq,Sk,D,causal", _cases(60, 21, "plain"))
+def test_single_sub_tile_launches(wt, B, H, Hkv, Sq, Sk, D, causal):
+    check_launch(wt, B, H, Hkv, Sq, Sk, D, causal, one=True)
+
+
+@pytest.mark.parametrize("B,H,Hkv,Sq,Sk,D,causal,n_splits", _cases(40, 22, "split"))
+def test_single_sub_tile_split_kv_launches(wt, B, H, Hkv, Sq, Sk, D, causal, n_splits):
+    check_launch(wt, B, H, Hkv, Sq, Sk, D, causal, n_splits=n_splits, one=True)
+
+
 def _varlen_cases(n, seed):
     rng = np.random.default_rng(seed)
     out = []
@@ -206,6 +224,7 @@ def test_variable_length_launches(wt, B, H, Hkv, lq, lk, causal):
     cu_q = np.concatenate([[0], np.cumsum(lq)]).tolist()
     cu_k = np.concatenate([[0], np.cumsum(lk)]).tolist()
     check_launch(wt, B, H, Hkv, max(lq), max(lk), 128, causal, cu_q=cu_q, cu_k=cu_k)
+    check_launch(wt, B, H, Hkv, max(lq), max(lk), 128, causal, cu_q=cu_q, cu_k=cu_k, one=True)
 
 
 def test_the_five_configurations_and_the_papers_shape(wt):

@@ -21,6 +21,8 @@ struct WtTile {
 
 namespace {
 
+bool g_one_subtile = false;  // plan launches for the single-sub-tile kernel (128-row tiles)
+
 struct Launch {
     ave::FwdParams p{};
     bool causal, split, varlen;
@@ -46,7 +48,7 @@ bool make_launch(Launch &L, int B, int H, int Hkv, int Sq, int Sk, int D, int ca
     }
     L.p.cu_q = cu_q;
     L.p.cu_k = cu_k;
-    return ave::plan_work_tiles(L.p, B, H, Hkv, Sq, Sk, D, L.causal, L.split, n_splits, kps, rows_per_head);
+    return ave::plan_work_tiles(L.p, B, H, Hkv, Sq, Sk, D, L.causal, L.split, n_splits, kps, rows_per_head, g_one_subtile);
 }
 
 template <bool CAUSAL, bool SPLIT, bool VARLEN>
@@ -72,6 +74,9 @@ void decode_all(const Launch &L, WtTile *out) {
 }  // namespace
 
 extern "C" {
+
+// Plan for the single-sub-tile kernel (nonzero) or the two-sub-tile kernel (zero, the default).
+void wt_set_one_subtile(int on) { g_one_subtile = on != 0; }
 
 // n_splits = 0: the ordinary forward; > 0: a split-KV launch.  varlen != 0: cu_q / cu_k are host arrays of
 // B + 1 offsets and Sq / Sk the longest sequences.  Returns 0, or 1 if the grid does not fit.
