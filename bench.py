@@ -48,6 +48,7 @@ L2_BYTES = 126e6
 PER_WORKLOAD_DEFAULT = [
     "c1_tiny", "c2_mha_prefill", "c3_gqa_prefill", "c4_long_context", "c5_wide_noncausal",
     "paper_gqa_n1024", "paper_gqa_n2048", "paper_gqa_n4096", "paper_gqa_n8192", "paper_gqa_n16384",
+    "d192_gqa_prefill", "d256_gqa_prefill",
     "decode_mha_b8_k8192", "decode_gqa_b8_k16384", "decode_gqa_b1_k65536", "decode_gqa_b64_k4096",
     "gemm_n4096", "gemm_n8192", "gemm_n16384",
 ]

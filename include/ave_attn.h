@@ -50,7 +50,7 @@ typedef enum {
     AVE_OK = 0,
     AVE_ERR_NULL_POINTER = 1,       /* q, k, v, o or lse is NULL */
     AVE_ERR_BAD_SHAPE = 2,          /* a size <= 0, H % Hkv != 0, or a size beyond the limits below */
-    AVE_ERR_UNSUPPORTED_D = 3,      /* D not a multiple of 8 in [8, 128] (split-KV calls: not 64 or 128) */
+    AVE_ERR_UNSUPPORTED_D = 3,      /* D not a multiple of 8 in [8, 256] (split-KV calls: not 64 or 128) */
     AVE_ERR_MISALIGNED = 4,         /* q, k, v, o not 16-byte aligned, or lse not 4-byte aligned */
     AVE_ERR_BAD_SCALE = 5,          /* scale is NaN or infinite (zero and negative values are allowed) */
     AVE_ERR_UNSUPPORTED_DEVICE = 6, /* the current device is not compute capability 10.x */
@@ -69,10 +69,10 @@ typedef enum {
  *   v   bf16 [B, Hkv, Sk, D]   read
  *   o   bf16 [B, H,   Sq, D]   written
  *   lse fp32 [B, H,   Sq]      written
- * Limits: D a multiple of 8, 8 <= D <= 128 (the kernels compute with D rounded
- * up to 64 or 128: the loads zero-fill the extra columns, the stores clip them,
- * so D = 96 costs what D = 128 costs); H % Hkv == 0; Sq, Sk < 2^31 / 2;
- * B * H < 2^31.
+ * Limits: D a multiple of 8, 8 <= D <= 256 (the kernels compute with D rounded
+ * up to 64, 128 or 256: the loads zero-fill the extra columns, the stores clip
+ * them, so D = 96 costs what D = 128 costs and D = 192 what D = 256 costs);
+ * H % Hkv == 0; Sq, Sk < 2^31 / 2; B * H < 2^31.
  * causal: 0 = every key visible, nonzero = bottom-right aligned causal mask.
  * scale: multiplies Q K^T before the softmax (callers normally pass 1/sqrt(D)).
  * stream: a cudaStream_t; NULL is the legacy default stream.

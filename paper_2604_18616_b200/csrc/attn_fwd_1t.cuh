@@ -20,6 +20,10 @@
 //
 // TMEM columns (256 per CTA): S [0,128), O [128,128+D); P (bf16 pairs) overwrites the first 64
 // columns of S once a thread holds its whole score row in registers.
+//
+// The same kernel serves head dimensions above 128 (instantiated for D = 256; 136..248 run it on tensor maps
+// of the true width, zero-filled): O then needs 256 TMEM columns, so a second sub-tile has no room, the CTA
+// allocates all 512 columns and, with 64 KB each for the Q, K and V tiles, has an SM to itself.
 #pragma once
 
 #include <type_traits>
@@ -36,10 +40,12 @@ struct OneCfg {
     static constexpr int kTileBytes = BM * D * 2;            // the Q tile, a K tile or a V tile
     static constexpr int kBoxBytes = BM * 64 * 2;            // one 64-column TMA box (128 rows x 128 B)
     static constexpr int kBoxes = D / 64;
-    static constexpr int kStages = (D == 128) ? 2 : 4;       // ring slots, K and V tiles alternate (two CTAs must fit an SM)
+    static constexpr int kStages = (D >= 128) ? 2 : 4;       // ring slots, K and V tiles alternate (two CTAs must fit an SM)
     static constexpr int kSmemBytes = kTileBytes * (1 + kStages) + 1024;
-    static_assert(2 * (kSmemBytes + 2048) <= 228 * 1024, "two CTAs do not fit the shared memory of an SM");
-    static constexpr uint32_t kTmemCols = 256;
+    static constexpr int kCtasPerSm = (D <= 128) ? 2 : 1;
+    static_assert(kCtasPerSm * (kSmemBytes + 2048) <= 228 * 1024, "the CTAs do not fit the shared memory of an SM");
+    static constexpr uint32_t kTmemCols = (D <= 128) ? 256 : 512;
+    static_assert(128 + D <= int(kTmemCols), "S and O do not fit the TMEM allocation");
     static constexpr uint32_t kColS = 0, kColO = 128;
     static constexpr int kRegsLight = 48;                    // producer / MMA / scheduler warpgroup
     static constexpr int kRegsSoftmax = 208;                 // softmax warpgroup

@@ -140,7 +140,7 @@ int validate(const void *q, const void *k, const void *v, const void *o, const v
     if (H % Hkv != 0) return AVE_ERR_BAD_SHAPE;
     if (Sq >= (1 << 30) || Sk >= (1 << 30)) return AVE_ERR_BAD_SHAPE;
     if ((long long)B * H >= (1ll << 31)) return AVE_ERR_BAD_SHAPE;
-    if (D < 8 || D > 128 || D % 8 != 0) return AVE_ERR_UNSUPPORTED_D;
+    if (D < 8 || D > 256 || D % 8 != 0) return AVE_ERR_UNSUPPORTED_D;
     const long long n_qblk = (Sq + ave::BM - 1) / ave::BM;
     if (n_qblk * B * H >= (1ll << 31)) return AVE_ERR_BAD_SHAPE;
     return -1;  // shape checks passed; pointer/scale checks follow
@@ -311,7 +311,8 @@ int launch_attention(const void *q, const void *k, const void *v, void *o, float
     const Strides sv = layout ? layout[2] : varlen ? token_major(Hkv, rows_k) : contiguous_strides(Hkv, Sk, D);
     const Strides so = layout ? layout[3] : varlen ? token_major(H, rows_q) : contiguous_strides(H, Sq, D);
     const bool split = o_partial != nullptr;
-    const bool one = use_one_subtile(B, H, Hkv, Sq, Sk, causal, split, varlen != nullptr);
+    // a head dimension above 128 leaves no TMEM for a second sub-tile: only the single-sub-tile kernel has it
+    const bool one = D > 128 || use_one_subtile(B, H, Hkv, Sq, Sk, causal, split, varlen != nullptr);
     CUtensorMap tq, tk, tv, to;
     if (!encode_map(&tq, q, D, rows_q, H, n_batch, sq, ave::BM)) return AVE_ERR_CUDA;
     if (!one && !encode_map(&to, o, D, rows_q, H, n_batch, so, ave::WsCfg<128>::kOutBoxRows)) return AVE_ERR_CUDA;
@@ -328,13 +329,18 @@ int launch_attention(const void *q, const void *k, const void *v, void *o, float
     p.cu_q = varlen ? varlen->cu_q : nullptr;
     p.cu_k = varlen ? varlen->cu_k : nullptr;
     p.lse_stride_h = varlen ? varlen->total_q : 0;
-    const int Dk = D <= 64 ? 64 : 128;  // the kernel's head dimension: TMA zero-fills the columns beyond D
+    const int Dk = D <= 64 ? 64 : D <= 128 ? 128 : 256;  // the kernel's head dimension: TMA zero-fills the columns beyond D
     if (!ave::plan_work_tiles(p, B, H, Hkv, Sq, Sk, D, causal != 0, split, n_splits, keys_per_split, rows_per_head, one))
         return AVE_ERR_BAD_SHAPE;
     p.o_partial = o_partial;
     p.lse_partial = lse_partial;
     p.scale_log2 = scale * 1.4426950408889634f;
 
+    if (one && Dk == 256) {  // (the split-KV entry points take 64 or 128 only)
+        if (varlen)
+            return causal ? launch_1t<256, true, false, true>(tq, tk, tv, p, s) : launch_1t<256, false, false, true>(tq, tk, tv, p, s);
+        return causal ? launch_1t<256, true, false>(tq, tk, tv, p, s) : launch_1t<256, false, false>(tq, tk, tv, p, s);
+    }
     if (one) {
         if (split) {
             if (Dk == 128)
@@ -710,7 +716,7 @@ const char *ave_attn_strerror(int status) {
         case AVE_OK: return "ok";
         case AVE_ERR_NULL_POINTER: return "a required pointer is NULL";
         case AVE_ERR_BAD_SHAPE: return "bad shape: sizes must be positive, H a multiple of Hkv, and within limits";
-        case AVE_ERR_UNSUPPORTED_D: return "unsupported head dimension (a multiple of 8 up to 128; 64 or 128 for the split-KV calls)";
+        case AVE_ERR_UNSUPPORTED_D: return "unsupported head dimension (a multiple of 8 up to 256; 64 or 128 for the split-KV calls)";
         case AVE_ERR_MISALIGNED: return "q, k, v, o must be 16-byte aligned and lse 4-byte aligned";
         case AVE_ERR_BAD_SCALE: return "scale is NaN or infinite";
         case AVE_ERR_UNSUPPORTED_DEVICE: return "the current CUDA device is not compute capability 10.x";

@@ -67,6 +67,12 @@ for _n in (1024, 2048, 4096, 8192, 16384):
         note="the paper's evaluation shape (LLaMA-3 70B prefill under 8-way TP)")
 
 
+# Head dimensions above 128 (the single-sub-tile kernel with 256 output columns in TMEM).
+WORKLOADS["d256_gqa_prefill"] = Workload("d256_gqa_prefill", 2, 32, 8, 4096, 4096, 256, True, 301,
+                                         note="causal grouped-query prefill, head dimension 256")
+WORKLOADS["d192_gqa_prefill"] = Workload("d192_gqa_prefill", 2, 32, 8, 4096, 4096, 192, True, 302,
+                                         note="causal grouped-query prefill, head dimension 192 (computed as 256)")
+
 # Decode: one new query token per sequence against a long key/value cache (the split-KV entry point);
 # bound by reading K and V once from HBM.
 for _name, _b, _h, _hkv, _sk, _seed in (("decode_mha_b8_k8192", 8, 32, 32, 8192, 201),

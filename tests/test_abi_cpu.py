@@ -66,7 +66,8 @@ def test_validation_order_before_any_cuda_call(lib):
     assert f(A, A, A, A, A, 1, 6, 4, 128, 128, 64, 0, 1.0) == binding.AVE_ERR_BAD_SHAPE      # H % Hkv
     assert f(A, A, A, A, A, 1, 2, 2, 1 << 30, 128, 64, 0, 1.0) == binding.AVE_ERR_BAD_SHAPE
     assert f(A, A, A, A, A, 1, 2, 2, 128, 128, 100, 0, 1.0) == binding.AVE_ERR_UNSUPPORTED_D
-    assert f(A, A, A, A, A, 1, 2, 2, 128, 128, 256, 0, 1.0) == binding.AVE_ERR_UNSUPPORTED_D
+    assert f(A, A, A, A, A, 1, 2, 2, 128, 128, 264, 0, 1.0) == binding.AVE_ERR_UNSUPPORTED_D
+    assert f(A, A, A, A, A, 1, 2, 2, 128, 128, 4, 0, 1.0) == binding.AVE_ERR_UNSUPPORTED_D
     assert f(A + 8, A, A, A, A, 1, 2, 2, 128, 128, 64, 0, 1.0) == binding.AVE_ERR_MISALIGNED
     assert f(A, A, A, A + 2, A, 1, 2, 2, 128, 128, 64, 0, 1.0) == binding.AVE_ERR_MISALIGNED
     assert f(A, A, A, A, A + 2, 1, 2, 2, 128, 128, 64, 0, 1.0) == binding.AVE_ERR_MISALIGNED

@@ -220,3 +220,33 @@ def test_full_size_configs_sampled_rows(name, n_random):
     # property that holds at any size: softmax weights are a convex combination of V rows
     vmax = v.float().abs().amax().item()
     assert o.float().abs().max().item() <= vmax * (1 + 2 ** -7)
+
+
+WIDE_SHAPES = [
+    # B, H, Hkv, Sq, Sk, D, causal : head dimensions above 128 (computed with 256 output columns)
+    (1, 2, 2, 1, 1, 256, True),
+    (1, 2, 1, 130, 130, 256, True),
+    (2, 4, 2, 257, 300, 192, True),
+    (1, 3, 3, 128, 513, 256, False),
+    (1, 4, 1, 300, 300, 136, True),
+    (1, 2, 2, 400, 130, 200, True),     # Sq > Sk: leading rows see no key
+    (1, 8, 2, 7, 777, 248, False),
+]
+
+
+@pytest.mark.parametrize("B,H,Hkv,Sq,Sk,D,causal", WIDE_SHAPES)
+def test_head_dimensions_above_128(B, H, Hkv, Sq, Sk, D, causal):
+    q, k, v = rand_qkv(D * 31 + Sq, B, H, Hkv, Sq, Sk, D)
+    parity.check_full(q, k, v, causal, 1.0 / math.sqrt(D), "wide head %s" % ((B, H, Hkv, Sq, Sk, D, causal),))
+
+
+@pytest.mark.parametrize("name", ["d192_gqa_prefill", "d256_gqa_prefill"])
+def test_wide_head_workloads_sampled_rows(name):
+    """Full-size runs of the wide-head workloads: tile-edge rows of every (b, h) plus random rows, and two runs
+    bit for bit equal."""
+    w = inputs.get(name)
+    q, k, v = inputs.make_inputs(w)
+    o, lse = parity.run_gpu(q, k, v, w.causal, w.scale)
+    o2, lse2 = parity.run_gpu(q, k, v, w.causal, w.scale)
+    assert torch.equal(o, o2) and torch.equal(lse, lse2)
+    parity.check_rows(o, lse, q, k, v, inputs.sample_rows(w, 512), w.causal, w.scale, name)

@@ -30,6 +30,8 @@ def _check(o_view, lse, q, k, v, causal, scale, what):
     (2, 4, 4, 300, 300, 128, True),     # several tiles and a ragged tail
     (1, 8, 2, 257, 513, 64, True),      # GQA, Sq != Sk, D = 64
     (2, 3, 1, 128, 700, 128, False),    # non-causal, one KV head
+    (1, 4, 2, 200, 330, 256, True),     # head dimension 256 (the single-sub-tile kernel)
+    (1, 2, 2, 130, 130, 192, False),
 ])
 def test_sequence_head_d_layout(B, H, Hkv, Sq, Sk, D, causal):
     """Storage (B, S, H, D) as in the paper's Fig. 1; the tensors handed over are permuted views."""

@@ -52,7 +52,7 @@ def _run_and_check(lens_q, lens_k, H, Hkv, D, causal, seed, max_pad=0):
 
 
 @pytest.mark.parametrize("causal", [False, True])
-@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("D", [64, 128, 192, 256])
 def test_self_attention_lengths_on_and_off_tile_edges(causal, D):
     lens = [256, 1, 127, 300, 128, 513, 32, 129]
     _run_and_check(lens, lens, 4, 2, D, causal, 31)
