@@ -54,10 +54,13 @@ struct WsCfg {
     static constexpr int kTileConsumers = 10;               // producer + MMA + 8 softmax warps read each tile id
 };
 
-// Rescale O only when the running maximum moved by more than this many
-// powers of two; until then probabilities are taken relative to a stale
-// maximum (at most 2^8 too large), which the final division by l undoes.
-constexpr float kRescaleThreshold = 8.0f;
+// Rescale O only when the running maximum moved by more than this many powers of two; until then
+// probabilities are taken relative to a stale maximum (at most 2^32 too large), which the final division by l
+// undoes.  Nothing is lost by a large threshold: P is rounded to bf16, which has fp32's exponent range, and
+// scaling every probability of a row by one factor leaves the relative rounding errors of P, l and O as they
+// are; l and O stay below 2^32 * Sk * max|V|, far from fp32's limit.  With peaked rows (the long-context
+// configuration) a threshold of 8 made some row of a warp rescale in most steps; measured -5.6 % there.
+constexpr float kRescaleThreshold = 32.0f;
 
 // Of every 8 consecutive pairs of probabilities, the pairs whose bit is set
 // here are exponentiated on the FMA pipe (exp2_fma_pipe) instead of the
@@ -68,13 +71,13 @@ constexpr float kRescaleThreshold = 8.0f;
 constexpr unsigned kFmaPipeExpMask = AVE_FMA_EXP_MASK;
 
 // Trace builds record the role timeline of two consecutive tiles of a CTA, starting at this one (0 = its first);
-// the second tile's steps follow at iteration index 32.
+// the second tile's steps follow at iteration index 32 (steps beyond the 27th of a tile share its slot).
 #ifndef AVE_TRACE_TILE
 #define AVE_TRACE_TILE 0
 #endif
 constexpr int kTraceTile = AVE_TRACE_TILE;
 __device__ __forceinline__ bool traced(int n) { return unsigned(n - kTraceTile) < 2u; }
-__device__ __forceinline__ int trace_it(int n, int j) { return (n - kTraceTile) * 32 + (j < 30 ? j : 29); }
+__device__ __forceinline__ int trace_it(int n, int j) { return (n - kTraceTile) * 32 + (j < 28 ? j : 27); }  // 28, 30: per-tile stamps
 
 template <int N>
 __device__ __forceinline__ void setmaxnreg_inc() {

@@ -53,10 +53,12 @@ def events(stamps):
                     text = "the CTA's tile number %d starts" % it
                     who = "MMA"
                 elif j == 28:
-                    text = "T%d %s" % (tile, ["tile loop start", "Q0 issue", "Q1 issue", "all loads issued", "next tile known"][sl])
+                    lab = ["tile loop start", "Q0 issue", "Q1 issue", "all loads issued", "next tile known"]
+                    text = "T%d %s" % (tile, lab[sl] if sl < len(lab) else "stamp %d" % sl)
                     who = NAMES[role]
                 elif j == 30:
-                    text = "T%d %s" % (tile, ["epilogue: wait for O", "epilogue: O ready", "epilogue done", "next tile known"][sl])
+                    lab = ["epilogue: wait for O", "epilogue: O ready", "epilogue done", "next tile known"]
+                    text = "T%d %s" % (tile, lab[sl] if sl < len(lab) else "stamp %d" % sl)
                     who = NAMES[role]
                 else:
                     lab = LABELS[role]
