@@ -20,6 +20,8 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "ave_oracle.c")
 _HDR = os.path.join(_HERE, "ave_oracle.h")
+_SRC_MOE = os.path.join(_HERE, "ave_oracle_moe.c")
+_HDR_MOE = os.path.join(_HERE, "ave_oracle_moe.h")
 _LIB = os.path.join(_HERE, "libave_oracle.so")
 _lock = threading.Lock()
 _lib = None
@@ -27,11 +29,11 @@ _lib = None
 
 def build(force: bool = False) -> str:
     """Compile ``ave_oracle.c`` with gcc into ``libave_oracle.so`` beside it."""
-    newest_src = max(os.path.getmtime(_SRC), os.path.getmtime(_HDR))
+    newest_src = max(os.path.getmtime(f) for f in (_SRC, _HDR, _SRC_MOE, _HDR_MOE))
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < newest_src:
         tmp = _LIB + ".tmp%d" % os.getpid()
         cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared",
-               "-Wall", "-Wextra", "-o", tmp, _SRC, "-lm"]
+               "-Wall", "-Wextra", "-o", tmp, _SRC, _SRC_MOE, "-lm"]
         subprocess.run(cmd, check=True, cwd=_HERE)
         os.replace(tmp, _LIB)
     return _LIB
@@ -56,6 +58,20 @@ def _load():
             lib.ave_oracle_gemm_tn.restype = ctypes.c_int
             lib.ave_oracle_gemm_tn_entries.argtypes = [u16p, u16p, i64p, ctypes.c_int64, f64p] + [ctypes.c_int] * 3
             lib.ave_oracle_gemm_tn_entries.restype = ctypes.c_int
+            u8p = ctypes.POINTER(ctypes.c_uint8)
+            f32p = ctypes.POINTER(ctypes.c_float)
+            i32p = ctypes.POINTER(ctypes.c_int32)
+            lib.ave_oracle_e4m3_decode.argtypes = [ctypes.c_uint8]
+            lib.ave_oracle_e4m3_decode.restype = ctypes.c_double
+            lib.ave_oracle_e4m3_encode.argtypes = [ctypes.c_float]
+            lib.ave_oracle_e4m3_encode.restype = ctypes.c_uint8
+            lib.ave_oracle_quant_groups.argtypes = [f32p, ctypes.c_int64, u8p, f32p]
+            lib.ave_oracle_quant_groups.restype = ctypes.c_int
+            moe = [u8p, f32p, u8p, f32p, u8p, f32p, i32p, f32p]
+            lib.ave_oracle_moe_fwd.argtypes = moe + [f64p, u8p, f32p] + [ctypes.c_int] * 5
+            lib.ave_oracle_moe_fwd.restype = ctypes.c_int
+            lib.ave_oracle_moe_rows.argtypes = moe + [i64p, ctypes.c_int64, f64p] + [ctypes.c_int] * 5
+            lib.ave_oracle_moe_rows.restype = ctypes.c_int
             lib.ave_oracle_threads.argtypes = []
             lib.ave_oracle_threads.restype = ctypes.c_int
             _lib = lib
@@ -173,3 +189,68 @@ def gemm_tn_entries(a, b, idx):
     if rc != 0:
         raise ValueError("ave_oracle_gemm_tn_entries rejected its arguments (rc=%d)" % rc)
     return out
+
+
+# ------------------------------------------------------------------ fused MoE (ave_oracle_moe.h)
+def e4m3_decode(code: int) -> float:
+    return float(_load().ave_oracle_e4m3_decode(int(code) & 0xFF))
+
+
+def e4m3_encode(x: float) -> int:
+    return int(_load().ave_oracle_e4m3_encode(float(x)))
+
+
+def quant_groups(a):
+    """Quantise fp32 values in groups of 128 along the last axis: (codes uint8, scales fp32)."""
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    if a.shape[-1] % 128:
+        raise ValueError("the last dimension must be a multiple of 128")
+    codes = np.empty(a.shape, np.uint8)
+    scales = np.empty(a.shape[:-1] + (a.shape[-1] // 128,), np.float32)
+    rc = _load().ave_oracle_quant_groups(_ptr(a, ctypes.c_float), a.size // 128, _ptr(codes, ctypes.c_uint8),
+                                         _ptr(scales, ctypes.c_float))
+    if rc != 0:
+        raise ValueError("ave_oracle_quant_groups rejected its arguments")
+    return codes, scales
+
+
+def _moe_args(xq, sx, w13q, s13, w2q, s2, ids, wts):
+    xq, w13q, w2q = (np.ascontiguousarray(a, dtype=np.uint8) for a in (xq, w13q, w2q))
+    sx, s13, s2, wts = (np.ascontiguousarray(a, dtype=np.float32) for a in (sx, s13, s2, wts))
+    ids = np.ascontiguousarray(ids, dtype=np.int32)
+    T, C = xq.shape
+    E, F2, C2 = w13q.shape
+    F = F2 // 2
+    K = ids.shape[1]
+    if C2 != C or w2q.shape != (E, C, F) or sx.shape != (T, C // 128) or s13.shape != (E, F2 // 128, C // 128) or \
+            s2.shape != (E, C // 128, F // 128) or wts.shape != (T, K) or ids.shape[0] != T:
+        raise ValueError("inconsistent MoE shapes")
+    ptrs = [_ptr(xq, ctypes.c_uint8), _ptr(sx, ctypes.c_float), _ptr(w13q, ctypes.c_uint8), _ptr(s13, ctypes.c_float),
+            _ptr(w2q, ctypes.c_uint8), _ptr(s2, ctypes.c_float), _ptr(ids, ctypes.c_int32), _ptr(wts, ctypes.c_float)]
+    keep = (xq, sx, w13q, s13, w2q, s2, ids, wts)
+    return ptrs, keep, (T, C, F, E, K)
+
+
+def moe_fwd(xq, sx, w13q, s13, w2q, s2, ids, wts, return_intermediate: bool = False):
+    """y [T, C] in float64 (and the requantised intermediates aq [T,K,F] uint8, sa [T,K,F/128] fp32)."""
+    ptrs, keep, (T, C, F, E, K) = _moe_args(xq, sx, w13q, s13, w2q, s2, ids, wts)
+    y = np.empty((T, C), np.float64)
+    aq = np.empty((T, K, F), np.uint8) if return_intermediate else None
+    sa = np.empty((T, K, F // 128), np.float32) if return_intermediate else None
+    rc = _load().ave_oracle_moe_fwd(*ptrs, _ptr(y, ctypes.c_double),
+                                    _ptr(aq, ctypes.c_uint8) if return_intermediate else None,
+                                    _ptr(sa, ctypes.c_float) if return_intermediate else None, T, C, F, E, K)
+    if rc != 0:
+        raise ValueError("ave_oracle_moe_fwd rejected its arguments (rc=%d)" % rc)
+    return (y, aq, sa) if return_intermediate else y
+
+
+def moe_rows(xq, sx, w13q, s13, w2q, s2, ids, wts, tokens):
+    """Oracle rows of y for selected tokens: [n, C] float64."""
+    ptrs, keep, (T, C, F, E, K) = _moe_args(xq, sx, w13q, s13, w2q, s2, ids, wts)
+    tok = np.ascontiguousarray(np.asarray(tokens, dtype=np.int64).reshape(-1))
+    y = np.empty((tok.shape[0], C), np.float64)
+    rc = _load().ave_oracle_moe_rows(*ptrs, _ptr(tok, ctypes.c_int64), tok.shape[0], _ptr(y, ctypes.c_double), T, C, F, E, K)
+    if rc != 0:
+        raise ValueError("ave_oracle_moe_rows rejected its arguments (rc=%d)" % rc)
+    return y

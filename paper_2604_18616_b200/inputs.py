@@ -173,3 +173,68 @@ def make_gemm_inputs(M: int, N: int, K: int, seed: int):
     a = torch.randn((M, K), generator=g, dtype=torch.float32).to(torch.bfloat16)
     b = torch.randn((N, K), generator=g, dtype=torch.float32).to(torch.bfloat16)
     return a, b
+
+
+# ------------------------------------------------------------------ fused MoE (block-quantised FP8)
+@dataclass(frozen=True)
+class MoeWorkload:
+    """The paper's fused-MoE configuration (Section 9): model dimension C, intermediate dimension F, top-k K,
+    E experts on this GPU; T tokens whose K routed experts all live on this GPU."""
+    name: str
+    T: int
+    C: int = 7168
+    F: int = 2048
+    E: int = 32
+    K: int = 4
+    seed: int = 400
+
+
+MOE_WORKLOADS = {n: MoeWorkload(n, t, seed=400 + i) for i, (n, t) in enumerate(
+    (("moe_t256", 256), ("moe_t1024", 1024), ("moe_t4096", 4096), ("moe_t8192", 8192), ("moe_t16384", 16384)))}
+
+
+def _fp8_codes(g: torch.Generator, shape, group_axis_len: int):
+    """Random E4M3 bit patterns shaped like block-quantised Gaussian data: the exponent field is drawn from a
+    fixed table of weights (most values within a factor of 8 below the block maximum), mantissa and sign
+    uniformly; the first element of every group of 128 along the last axis is the block maximum (+-448, code
+    0x7e), as it is after scaling a block by its largest magnitude.  No NaN pattern is produced.  Bit patterns
+    only: nothing here evaluates the format."""
+    n = 1
+    for d in shape:
+        n *= d
+    weights = torch.zeros(16)
+    weights[15], weights[14], weights[13], weights[12], weights[11] = 0.10, 0.32, 0.28, 0.15, 0.08
+    weights[10], weights[9], weights[8] = 0.04, 0.02, 0.01
+    expo = torch.multinomial(weights, n, replacement=True, generator=g).to(torch.uint8)
+    mant = torch.randint(0, 8, (n,), generator=g, dtype=torch.uint8)
+    mant = torch.where((expo == 15) & (mant == 7), torch.zeros_like(mant), mant)   # 0x7f would be NaN
+    sign = torch.randint(0, 2, (n,), generator=g, dtype=torch.uint8) << 7
+    codes = (sign | (expo << 3) | mant).reshape(shape)
+    lead = codes[..., ::group_axis_len]
+    codes[..., ::group_axis_len] = (lead & 0x80) | 0x7E
+    return codes.contiguous()
+
+
+def make_moe_inputs(w: MoeWorkload):
+    """(xq u8 [T,C], sx f32 [T,C/128], w13q u8 [E,2F,C], s13 f32 [E,2F/128,C/128], w2q u8 [E,C,F],
+    s2 f32 [E,C/128,F/128], ids i32 [T,K], wts f32 [T,K]) as CPU tensors.  Scales are drawn so that the
+    dequantised activations look like N(0,1) data and the dequantised weights like N(0, 1/fan_in) data; every
+    token gets K distinct experts and positive routing weights that sum to one."""
+    g = torch.Generator(device="cpu")
+    g.manual_seed(w.seed)
+    T, C, F, E, K = w.T, w.C, w.F, w.E, w.K
+    xq = _fp8_codes(g, (T, C), 128)
+    sx = (0.8 + 0.4 * torch.rand((T, C // 128), generator=g)) * (2.8 / 448.0)
+    w13q = _fp8_codes(g, (E, 2 * F, C), 128)
+    s13 = (0.8 + 0.4 * torch.rand((E, 2 * F // 128, C // 128), generator=g)) * (2.8 / 448.0 / math.sqrt(C))
+    w2q = _fp8_codes(g, (E, C, F), 128)
+    s2 = (0.8 + 0.4 * torch.rand((E, C // 128, F // 128), generator=g)) * (2.8 / 448.0 / math.sqrt(F))
+    ids = torch.stack([torch.randperm(E, generator=g)[:K] for _ in range(T)]).to(torch.int32)
+    raw = 0.1 + torch.rand((T, K), generator=g)
+    wts = (raw / raw.sum(dim=1, keepdim=True)).to(torch.float32)
+    return xq, sx.float(), w13q, s13.float(), w2q, s2.float(), ids, wts
+
+
+def moe_flops(w: MoeWorkload) -> float:
+    """Counted FLOPs: 2 * T * K * (2F*C + C*F)."""
+    return 2.0 * w.T * w.K * (2.0 * w.F * w.C + 1.0 * w.C * w.F)
