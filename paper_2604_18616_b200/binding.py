@@ -73,6 +73,10 @@ def lib() -> ctypes.CDLL:
         L.ave_gemm_bf16_tn.restype = ci
         L.ave_gemm_bf16_nn.argtypes = [vp, vp, vp, ci, ci, ci, vp]
         L.ave_gemm_bf16_nn.restype = ci
+        L.ave_moe_fused_fwd.argtypes = [vp] * 9 + [ci] * 5 + [vp, ctypes.c_size_t, vp]
+        L.ave_moe_fused_fwd.restype = ci
+        L.ave_moe_workspace_bytes.argtypes = [ci] * 5
+        L.ave_moe_workspace_bytes.restype = ctypes.c_size_t
         L.ave_attn_device_status.argtypes = [ctypes.POINTER(ctypes.c_uint)]
         L.ave_attn_device_status.restype = ci
         L.ave_attn_launch_count.argtypes = []
@@ -382,3 +386,38 @@ def ave_gemm_bf16_nn(a, b, c=None, stream=None):
     if st != AVE_OK:
         raise AveAttnError(st, "ave_gemm_bf16_nn")
     return c
+
+
+def moe_workspace_bytes(T, C, F, E, K) -> int:
+    return int(lib().ave_moe_workspace_bytes(T, C, F, E, K))
+
+
+def ave_moe_fused_fwd(xq, sx, w13q, s13, w2q, s2, ids, wts, y=None, workspace=None, stream=None):
+    """y [T, C] bf16 = fused block-quantised FP8 MoE layer on the tensors' CUDA device.
+
+    xq u8 [T,C], sx f32 [T,C/128], w13q u8 [E,2F,C], s13 f32 [E,2F/128,C/128], w2q u8 [E,C,F],
+    s2 f32 [E,C/128,F/128], ids i32 [T,K], wts f32 [T,K]: contiguous CUDA tensors.  ``workspace`` is a CUDA uint8
+    tensor of at least ``moe_workspace_bytes`` bytes (allocated here when not given)."""
+    for t, dt in ((xq, torch.uint8), (w13q, torch.uint8), (w2q, torch.uint8), (sx, torch.float32), (s13, torch.float32),
+                  (s2, torch.float32), (ids, torch.int32), (wts, torch.float32)):
+        if not (t.is_cuda and t.dtype == dt and t.is_contiguous()):
+            raise ValueError("MoE inputs must be contiguous CUDA tensors of the documented dtypes")
+    T, C = xq.shape
+    E, F2, C2 = w13q.shape
+    F = F2 // 2
+    K = ids.shape[1]
+    if C2 != C or tuple(w2q.shape) != (E, C, F) or tuple(ids.shape) != (T, K) or tuple(wts.shape) != (T, K):
+        raise ValueError("inconsistent MoE shapes")
+    if y is None:
+        y = torch.empty((T, C), dtype=torch.bfloat16, device=xq.device)
+    if workspace is None:
+        workspace = torch.empty(max(256, moe_workspace_bytes(T, C, F, E, K)), dtype=torch.uint8, device=xq.device)
+    with torch.cuda.device(xq.device):
+        st = lib().ave_moe_fused_fwd(
+            ctypes.c_void_p(xq.data_ptr()), ctypes.c_void_p(sx.data_ptr()), ctypes.c_void_p(w13q.data_ptr()),
+            ctypes.c_void_p(s13.data_ptr()), ctypes.c_void_p(w2q.data_ptr()), ctypes.c_void_p(s2.data_ptr()),
+            ctypes.c_void_p(ids.data_ptr()), ctypes.c_void_p(wts.data_ptr()), ctypes.c_void_p(y.data_ptr()),
+            T, C, F, E, K, ctypes.c_void_p(workspace.data_ptr()), ctypes.c_size_t(workspace.numel()), _stream_ptr(stream))
+    if st != AVE_OK:
+        raise AveAttnError(st, "ave_moe_fused_fwd")
+    return y

@@ -3,6 +3,7 @@
 // for the contract of every exported function.
 #include "../../include/ave_attn.h"
 #include "../../include/ave_gemm.h"
+#include "../../include/ave_moe.h"
 
 #include <atomic>
 #include <cmath>
@@ -16,6 +17,7 @@
 #include "attn_fwd_ws.cuh"
 #include "attn_fwd_1t.cuh"
 #include "gemm_bf16.cuh"
+#include "moe_fp8.cuh"
 
 // Scratch of ave_attn_fwd_splitkv_static: part of the device image, so every GPU that loads the
 // library holds it until exit.  In host code this name is only a handle for
@@ -508,9 +510,189 @@ int launch_gemm(const void *a, const void *b, void *c, int M, int N, int K, cuda
     return launch_gemm_tile<256, B_NMAJOR>(a, b, c, M, N, K, sms, s);
 }
 
+// E4M3 codes [d3, d2, rows, inner] (inner contiguous) as a 4-D map with boxes of 128 bytes x 128 rows, 128-byte
+// swizzle.  (Not cached: two encodes per GEMM of a layer call.)
+bool encode_map_u8(CUtensorMap *map, const void *base, long long inner, long long rows, long long d2) {
+    if (take_injected(g_inject_encode_failures)) {
+        t_last_cuda_error = int(CUDA_ERROR_INVALID_VALUE);
+        return false;
+    }
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return false;
+    cuuint64_t gdim[4] = {cuuint64_t(inner), cuuint64_t(rows), cuuint64_t(d2), 1};
+    cuuint64_t gstride[3] = {cuuint64_t(inner), cuuint64_t(inner) * cuuint64_t(rows), cuuint64_t(inner) * cuuint64_t(rows) * cuuint64_t(d2)};
+    cuuint32_t box[4] = {128, 128, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(base), gdim, gstride, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    g_map_encodes.fetch_add(1, std::memory_order_relaxed);
+    if (r != CUDA_SUCCESS) {
+        t_last_cuda_error = int(r);
+        return false;
+    }
+    return true;
+}
+
+// Scratch of one fused-MoE call, carved out of the caller's workspace (every part 256-byte aligned).
+struct MoeWorkspace {
+    long long rows_cap;  // rows of the sorted order, padding included: a multiple of 128
+    size_t xq_s, sx_s, ho, aq, sa, row_of, pair_of, w_s, expert_off, cursor, tile_expert, bad_id, total;
+};
+bool moe_layout(MoeWorkspace &w, int T, int C, int F, int E, int K) {
+    if (T <= 0 || C <= 0 || F <= 0 || E <= 0 || K <= 0 || C % 128 || F % 128 || E > 1024) return false;
+    const long long pairs = (long long)T * K;
+    if (pairs >= (1ll << 24)) return false;
+    w.rows_cap = 128 * ((pairs + 127) / 128 + E);  // sum over experts of ceil(rows / 128) tiles is at most this many
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        const size_t at = off;
+        off = (off + bytes + 255) & ~size_t(255);
+        return at;
+    };
+    const size_t rows = size_t(w.rows_cap);
+    w.xq_s = take(rows * C);
+    w.sx_s = take(rows * (C / 128) * 4);
+    // the up projection's result h [rows, 2F] is dead once the activations are requantised: the down projection's
+    // result o [rows, C] takes the same space
+    w.ho = take(rows * size_t(2 * F > C ? 2 * F : C) * 4);
+    w.aq = take(rows * F);
+    w.sa = take(rows * (F / 128) * 4);
+    w.row_of = take(size_t(pairs) * 4);
+    w.pair_of = take(rows * 4);
+    w.w_s = take(rows * 4);
+    w.expert_off = take(size_t(E + 1) * 4);
+    w.cursor = take(size_t(E) * 4);
+    w.tile_expert = take(rows / 128 * 4);
+    w.bad_id = take(4);
+    w.total = off;
+    return true;
+}
+
+int launch_moe_gemm(const void *a, long long rows, const float *a_scale, const void *b, const float *b_scale, int E,
+                    int N, int K, const int *tile_expert, const float *row_weight, float *out, int sms, cudaStream_t s) {
+    using Cfg = ave::MoeGemmCfg;
+    CUtensorMap ta, tb;
+    if (!encode_map_u8(&ta, a, K, rows, 1)) return AVE_ERR_CUDA;
+    if (!encode_map_u8(&tb, b, K, N, E)) return AVE_ERR_CUDA;
+    ave::MoeGemmParams p;
+    p.a_scale = a_scale;
+    p.b_scale = b_scale;
+    p.tile_expert = tile_expert;
+    p.row_weight = row_weight;
+    p.out = out;
+    p.tiles_m = int(rows / 128);
+    p.tiles_n = N / 128;
+    p.kb = K / 128;
+    p.N = N;
+    static PerDeviceOnce once;
+    const int st = prepare_kernel(ave::moe_gemm_fp8_kernel, Cfg::kSmemBytes, 0, once);
+    if (st != AVE_OK) return st;
+    if (take_injected(g_inject_launch_failures)) {
+        t_last_cuda_error = int(cudaErrorLaunchFailure);
+        return AVE_ERR_CUDA;
+    }
+    const long long n_tiles = (long long)p.tiles_m * p.tiles_n;
+    const unsigned grid = unsigned(n_tiles < sms ? n_tiles : sms);
+    ave::moe_gemm_fp8_kernel<<<dim3(grid), dim3(Cfg::kThreads), Cfg::kSmemBytes, s>>>(ta, tb, p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        t_last_cuda_error = int(e);
+        return AVE_ERR_CUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return AVE_OK;
+}
+
+// One of the layer's small kernels has been launched: count it or report the launch error.
+int after_small_launch() {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        t_last_cuda_error = int(e);
+        return AVE_ERR_CUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return AVE_OK;
+}
+
 }  // namespace
 
 extern "C" {
+
+size_t ave_moe_workspace_bytes(int T, int C, int F, int E, int K) {
+    MoeWorkspace w;
+    return moe_layout(w, T, C, F, E, K) ? w.total : 0;
+}
+
+int ave_moe_fused_fwd(const void *xq, const float *sx, const void *w13q, const float *s13, const void *w2q,
+                      const float *s2, const int *ids, const float *wts, void *y, int T, int C, int F, int E, int K,
+                      void *workspace, size_t workspace_bytes, void *stream) {
+    if (!xq || !sx || !w13q || !s13 || !w2q || !s2 || !ids || !wts || !y) return AVE_ERR_NULL_POINTER;
+    MoeWorkspace w;
+    if (!moe_layout(w, T, C, F, E, K)) return AVE_ERR_BAD_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(xq) | reinterpret_cast<uintptr_t>(w13q) | reinterpret_cast<uintptr_t>(w2q) |
+         reinterpret_cast<uintptr_t>(y)) & 15u)
+        return AVE_ERR_MISALIGNED;
+    if ((reinterpret_cast<uintptr_t>(sx) | reinterpret_cast<uintptr_t>(s13) | reinterpret_cast<uintptr_t>(s2) |
+         reinterpret_cast<uintptr_t>(ids) | reinterpret_cast<uintptr_t>(wts)) & 3u)
+        return AVE_ERR_MISALIGNED;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < w.total) return AVE_ERR_WORKSPACE;
+    int st = check_device();
+    if (st != AVE_OK) return st;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess || sms <= 0) {
+        t_last_cuda_error = int(e);
+        return AVE_ERR_CUDA;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint8_t *base = static_cast<uint8_t *>(workspace);
+    uint8_t *xq_s = base + w.xq_s;
+    float *sx_s = reinterpret_cast<float *>(base + w.sx_s);
+    float *ho = reinterpret_cast<float *>(base + w.ho);
+    uint8_t *aq = base + w.aq;
+    float *sa = reinterpret_cast<float *>(base + w.sa);
+    int *row_of = reinterpret_cast<int *>(base + w.row_of);
+    int *pair_of = reinterpret_cast<int *>(base + w.pair_of);
+    float *w_s = reinterpret_cast<float *>(base + w.w_s);
+    int *expert_off = reinterpret_cast<int *>(base + w.expert_off);
+    int *cursor = reinterpret_cast<int *>(base + w.cursor);
+    int *tile_expert = reinterpret_cast<int *>(base + w.tile_expert);
+    int *bad_id = reinterpret_cast<int *>(base + w.bad_id);
+    const int pairs = T * K;
+    const int rows = int(w.rows_cap);
+
+    // 1. sort the (token, k) pairs by expert
+    ave::moe_count_kernel<<<1, 1024, size_t(E) * sizeof(int), s>>>(ids, pairs, E, rows, expert_off, cursor, tile_expert,
+                                                                  pair_of, bad_id);
+    if ((st = after_small_launch()) != AVE_OK) return st;
+    ave::moe_scatter_kernel<<<(pairs + 255) / 256, 256, 0, s>>>(ids, pairs, E, expert_off, cursor, row_of, pair_of);
+    if ((st = after_small_launch()) != AVE_OK) return st;
+    // 2. the tokens' codes and scales in sorted order
+    ave::moe_gather_kernel<<<rows, 128, 0, s>>>(static_cast<const uint8_t *>(xq), sx, wts, pair_of, tile_expert, C, K, xq_s,
+                                               sx_s, w_s);
+    if ((st = after_small_launch()) != AVE_OK) return st;
+    // 3. up projection: h = x W13^T
+    st = launch_moe_gemm(xq_s, rows, sx_s, w13q, s13, E, 2 * F, C, tile_expert, nullptr, ho, sms, s);
+    if (st != AVE_OK) return st;
+    // 4. activation and requantisation
+    {
+        const long long warps = (long long)rows * (F / 128);
+        ave::moe_act_quant_kernel<<<unsigned((warps + 7) / 8), 256, 0, s>>>(ho, tile_expert, F, rows, aq, sa);
+        if ((st = after_small_launch()) != AVE_OK) return st;
+    }
+    // 5. down projection, weighted: o = w * (a W2^T)
+    st = launch_moe_gemm(aq, rows, sa, w2q, s2, E, C, F, tile_expert, w_s, ho, sms, s);
+    if (st != AVE_OK) return st;
+    // 6. every token's K rows summed
+    {
+        const long long n = (long long)T * (C / 4);
+        ave::moe_combine_kernel<<<unsigned((n + 255) / 256), 256, 0, s>>>(ho, row_of, T, C, K, static_cast<__nv_bfloat16 *>(y));
+        if ((st = after_small_launch()) != AVE_OK) return st;
+    }
+    return AVE_OK;
+}
 
 int ave_attn_fwd(const void *q, const void *k, const void *v, void *o, float *lse, int B, int H, int Hkv, int Sq,
                  int Sk, int D, int causal, float scale, void *stream) {

@@ -26,7 +26,7 @@ def declared_functions():
             continue
         text = open(os.path.join(inc, header)).read()
         text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-        names.update(re.findall(r"\b(ave_(?:attn|gemm)_\w+)\s*\(", text))
+        names.update(re.findall(r"\b(ave_(?:attn|gemm|moe)_\w+)\s*\(", text))
     return sorted(names)
 
 
@@ -35,7 +35,8 @@ def test_header_declares_the_expected_entry_points():
     for n in ("ave_attn_fwd", "ave_attn_fwd_strided", "ave_attn_fwd_varlen", "ave_attn_fwd_host", "ave_attn_host_workspace_bytes", "ave_attn_device_status",
               "ave_attn_fwd_splitkv", "ave_attn_splitkv_workspace_bytes",
               "ave_attn_launch_count", "ave_attn_strerror", "ave_attn_version", "ave_attn_last_cuda_error",
-              "ave_gemm_bf16_tn", "ave_gemm_bf16_nn"):
+              "ave_gemm_bf16_tn", "ave_gemm_bf16_nn", "ave_moe_fused_fwd", "ave_moe_workspace_bytes",
+              "ave_attn_select_kernel", "ave_attn_splitkv_default_splits", "ave_attn_selftest_wait_timeout"):
         assert n in names
 
 
@@ -164,3 +165,25 @@ def test_selftest_hooks_validate_their_arguments(lib):
     assert binding.lib().ave_attn_selftest_wait_timeout(5, None) == binding.AVE_ERR_BAD_SHAPE
     assert binding.lib().ave_attn_selftest_wait_timeout(40, None) == binding.AVE_ERR_BAD_SHAPE
     assert binding.tensor_map_encodes() >= 0
+
+
+def test_moe_validation_before_any_cuda_call(lib):
+    A = 4096
+    L = binding.lib()
+    vp = ctypes.c_void_p
+    def f(ptrs, T, C, F, E, K, ws=A, ws_bytes=1 << 40):
+        return L.ave_moe_fused_fwd(*[vp(p) for p in ptrs], T, C, F, E, K, vp(ws), ctypes.c_size_t(ws_bytes), vp(0))
+    ok = [A] * 9
+    assert f([0] + ok[1:], 4, 256, 128, 2, 2) == binding.AVE_ERR_NULL_POINTER
+    assert f(ok[:8] + [0], 4, 256, 128, 2, 2) == binding.AVE_ERR_NULL_POINTER
+    assert f(ok, 0, 256, 128, 2, 2) == binding.AVE_ERR_BAD_SHAPE
+    assert f(ok, 4, 250, 128, 2, 2) == binding.AVE_ERR_BAD_SHAPE          # C not a multiple of 128
+    assert f(ok, 4, 256, 100, 2, 2) == binding.AVE_ERR_BAD_SHAPE          # F not a multiple of 128
+    assert f(ok, 1 << 22, 256, 128, 2, 8) == binding.AVE_ERR_BAD_SHAPE    # T * K too large
+    assert f([A + 8] + ok[1:], 4, 256, 128, 2, 2) == binding.AVE_ERR_MISALIGNED
+    assert f(ok[:1] + [A + 2] + ok[2:], 4, 256, 128, 2, 2) == binding.AVE_ERR_MISALIGNED
+    assert f(ok, 4, 256, 128, 2, 2, ws=0) == binding.AVE_ERR_WORKSPACE
+    assert f(ok, 4, 256, 128, 2, 2, ws_bytes=16) == binding.AVE_ERR_WORKSPACE
+    n = binding.moe_workspace_bytes(4096, 7168, 2048, 32, 4)
+    rows = 128 * (4096 * 4 // 128 + 32)
+    assert n >= rows * (7168 + 7168 * 4 + 2048) and n % 256 == 0
