@@ -39,6 +39,8 @@ if ROOT not in sys.path:
 
 METRIC = "attention fwd TFLOP/s (bf16, causal=half FLOPs)"
 GEMM_METRIC = "gemm TFLOP/s (bf16, 2*M*N*K)"
+MOE_METRIC = "fused MoE TFLOP/s (fp8 e4m3 block-quantised, 2*T*K*(2F*C + C*F))"
+FP8_OVER_BF16 = 2.0                   # nominal ratio of the dense fp8 and bf16 tensor peaks (4.5 / 2.25 PFLOP/s)
 UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "c4_long_context"
 NOMINAL_BF16_TFLOPS = 2250.0          # vendor dense bf16 figure, context only
@@ -51,6 +53,7 @@ PER_WORKLOAD_DEFAULT = [
     "d192_gqa_prefill", "d256_gqa_prefill",
     "decode_mha_b8_k8192", "decode_gqa_b8_k16384", "decode_gqa_b1_k65536", "decode_gqa_b64_k4096",
     "gemm_n4096", "gemm_n8192", "gemm_n16384",
+    "moe_t1024", "moe_t4096", "moe_t16384",
 ]
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel, from profiler captures of the
 # kernel as committed; a workload whose kernel has changed since its capture is absent (reported as null).
@@ -295,7 +298,13 @@ def run_reference(args):
     steps, warm = max(1, args.steps), max(0, args.warmup)
     per_step = max(0.5, min(args.cpu_seconds, 150.0 / (steps + warm)))
     is_gemm = args.workload.startswith("gemm_n")
-    if is_gemm:
+    is_moe = args.workload.startswith("moe_t")
+    if is_moe:
+        mw = inputs.MOE_WORKLOADS[args.workload]
+        margs = inputs.make_moe_inputs(mw)
+        sample = lambda: cpu_baseline_moe(mw, margs, per_step)
+        config = {"workload": mw.name, "T": mw.T, "C": mw.C, "F": mw.F, "E": mw.E, "K": mw.K}
+    elif is_gemm:
         n = gemm_size(args.workload)
         a, b = inputs.make_gemm_inputs(n, n, n, seed=20)
         sample = lambda: cpu_baseline_gemm(a, b, per_step)
@@ -311,7 +320,7 @@ def run_reference(args):
     value = sum(r["value"] for r in recs) / len(recs)
     total = sum(r["seconds"] for r in recs)
     print(json.dumps({
-        "impl": "reference", "metric": GEMM_METRIC if is_gemm else METRIC, "value": value, "unit": UNIT,
+        "impl": "reference", "metric": GEMM_METRIC if is_gemm else MOE_METRIC if is_moe else METRIC, "value": value, "unit": UNIT,
         "n_gpus": args.gpus, "steps": steps, "warmup": warm, "ms_per_step": 1e3 * total / steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": config,
@@ -586,11 +595,108 @@ def gemm_leg(ctx, name, steps, warmup, headline):
     return rec
 
 
+def cpu_baseline_moe(w, args, target_seconds, y_gpu=None):
+    """The oracle on a bounded sample of tokens (each costs K * 3 * C * F multiply-adds in fp64)."""
+    import numpy as np
+    import oracle
+    from paper_2604_18616_b200 import inputs
+    a = [t.numpy() for t in args]
+    cores = oracle.threads()
+    probe = list(range(min(w.T, max(1, cores))))
+    t0 = time.perf_counter()
+    oracle.moe_rows(*a, tokens=probe)
+    t_probe = time.perf_counter() - t0
+    n = int(min(w.T, max(len(probe), len(probe) * target_seconds / max(t_probe, 1e-6))))
+    tok = np.unique(np.linspace(0, w.T - 1, n).astype(np.int64))
+    t0 = time.perf_counter()
+    y_ref = oracle.moe_rows(*a, tokens=tok)
+    dt = time.perf_counter() - t0
+    out = {"value": inputs.moe_flops(w) * len(tok) / w.T / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+           "sample": "%d of %d tokens of %s, evenly spread, %.1f s" % (len(tok), w.T, w.name, dt), "seconds": dt}
+    if y_gpu is not None:
+        got = y_gpu[tok].double().numpy()
+        rms = float(np.sqrt(np.mean(y_ref ** 2))) + 1e-30
+        err = np.abs(got - y_ref)
+        tight = 2.0 ** -7 * np.abs(y_ref) + 2e-3 * rms
+        one_step = float(a[7].max()) * 448.0 * float(a[5].max())
+        out["parity"] = {"tokens": int(len(tok)), "max_abs_y": float(err.max()), "rms_y": rms,
+                         "frac_outside_tight": float(np.mean(err > tight)), "nan_left": bool(np.isnan(got).any()),
+                         "tol": "all within 2^-7|y| + one E4M3 step of an intermediate; 99.8 % within 2^-7|y| + 2e-3 rms",
+                         "ok": bool(np.mean(err > tight) <= 2e-3 and np.all(err <= 2.0 ** -7 * np.abs(y_ref) + one_step)
+                                    and not np.isnan(got).any())}
+    return out
+
+
+def moe_leg(ctx, name, steps, warmup, headline):
+    torch = ctx.torch
+    from paper_2604_18616_b200 import binding, inputs
+    w = inputs.MOE_WORKLOADS[name]
+    args = inputs.make_moe_inputs(w)
+    d = [t.to(ctx.dev) for t in args]
+    y = torch.empty((w.T, w.C), dtype=torch.bfloat16, device=ctx.dev)
+    ws = torch.empty(binding.moe_workspace_bytes(w.T, w.C, w.F, w.E, w.K), dtype=torch.uint8, device=ctx.dev)
+    flops = inputs.moe_flops(w)
+
+    def step(i):
+        binding.ave_moe_fused_fwd(*d, y=y, workspace=ws, stream=ctx.stream)
+
+    for i in range(max(warmup, 3)):
+        step(i)
+    ctx.barrier()
+    n0 = binding.launch_count()
+    ms = timed_launches(torch, ctx.stream, step, steps, ctx.clocks, ctx.barrier)
+    launches = binding.launch_count() - n0
+    clocks = ctx.clocks.summary()
+    ctx.check_status("the timed region of " + name)
+    peak8 = ctx.peak * FP8_OVER_BF16
+    weight_bytes = w.E * 3 * w.C * w.F
+    rec = {"workload": name, "kind": "moe", "config": {"workload": name, "T": w.T, "C": w.C, "F": w.F, "E": w.E, "K": w.K},
+           "steps": steps, "us": 1e3 * ms / steps, "tflops": flops / (ms / steps * 1e-3) / 1e12,
+           "gpu_launches": int(launches), "clocks": clocks, "input_sets": 1,
+           "roofline": {"bound": "tensor", "achieved": flops / (ms / steps * 1e-3) / 1e12, "peak": peak8, "unit": UNIT,
+                        "peak_kind": "measured bf16 matmul rate x the nominal fp8/bf16 ratio of 2",
+                        "algorithmic_hbm_bytes": weight_bytes + w.T * w.C * 3, "kernels_per_step": 7},
+           "_ms": ms, "_flops": flops}
+    rec["roofline"]["frac"] = rec["roofline"]["achieved"] / peak8
+    rec["frac"] = rec["roofline"]["frac"]
+    y.fill_(float("nan"))
+    step(0)
+    ctx.check_status("the checked launch of " + name)
+    rec["_moe"], rec["_args"], rec["_y"] = w, args, y.cpu()
+    rec["input_sha256"] = {"xq": inputs.tensor_sha256(args[0])[:16], "ids": inputs.tensor_sha256(args[6])[:16]}
+    if headline:
+        e2e_steps = max(1, min(ctx.args.e2e_steps, steps))
+        # the activations and the routing come from the host every step; the weights stay resident (a layer's weights
+        # do not change between calls)
+        hx, hs, hi, hw = (args[i].pin_memory() for i in (0, 1, 6, 7))
+        hy = torch.empty((w.T, w.C), dtype=torch.bfloat16).pin_memory()
+
+        def e2e_step(i):
+            d[0].copy_(hx, non_blocking=True)
+            d[1].copy_(hs, non_blocking=True)
+            d[6].copy_(hi, non_blocking=True)
+            d[7].copy_(hw, non_blocking=True)
+            binding.ave_moe_fused_fwd(*d, y=y, workspace=ws, stream=ctx.stream)
+            hy.copy_(y, non_blocking=True)
+
+        for i in range(3):
+            e2e_step(i)
+        ctx.barrier()
+        e2e_ms = timed_launches(torch, ctx.stream, e2e_step, e2e_steps, ctx.clocks, ctx.barrier)
+        rec["_e2e"] = {"ms": e2e_ms, "steps": e2e_steps, "h2d": sum(args[i].numel() * args[i].element_size() for i in (0, 1, 6, 7)),
+                       "d2h": hy.numel() * 2, "result_equal_to_device_path": bool(torch.equal(hy, rec["_y"]))}
+    del d, ws
+    torch.cuda.empty_cache()
+    return rec
+
+
 def finish_record(rec, cpu_seconds, want_oracle):
     """Run the CPU-baseline leg of a record (oracle timing + comparison with the GPU rows) and drop the tensors."""
     if want_oracle:
         if rec["kind"] == "gemm":
             rec["cpu_baseline"] = cpu_baseline_gemm(rec["_a"], rec["_b"], cpu_seconds, rec["_c"])
+        elif rec["kind"] == "moe":
+            rec["cpu_baseline"] = cpu_baseline_moe(rec["_moe"], rec["_args"], cpu_seconds, rec["_y"])
         else:
             rec["cpu_baseline"] = cpu_baseline_attention(rec["_w"], rec["_q"], rec["_k"], rec["_v"], cpu_seconds,
                                                          rec["_o"], rec["_lse"], spread=False)
@@ -605,6 +711,8 @@ def run_leg(ctx, name, steps, warmup, headline=False):
     from paper_2604_18616_b200 import inputs
     if name.startswith("gemm_n"):
         return gemm_leg(ctx, name, steps, warmup, headline)
+    if name.startswith("moe_t"):
+        return moe_leg(ctx, name, steps, warmup, headline)
     w = inputs.get(name)
     if name.startswith("decode_"):
         return decode_leg(ctx, w, steps, warmup)
@@ -625,10 +733,13 @@ def run_ours(args):
         flops = head["_flops"]
         ms_per_step = ms_max / steps
         is_gemm = head["kind"] == "gemm"
+        is_moe = head["kind"] == "moe"
         finish_record(head, args.cpu_seconds, want_oracle)
         kernel_tf = head["tflops"]
         if head["kind"] == "splitkv_decode":
             roofline = dict(head["roofline"], traffic=NCU_DRAM_BYTES_PER_LAUNCH.get(args.workload), peak_kind=ctx.peak_kind)
+        elif is_moe:
+            roofline = dict(head["roofline"], traffic=NCU_DRAM_BYTES_PER_LAUNCH.get(args.workload))
         else:
             w = None if is_gemm else inputs.get(args.workload)
             roofline = {"bound": "tensor", "achieved": kernel_tf, "peak": ctx.peak, "unit": UNIT,
@@ -644,9 +755,10 @@ def run_ours(args):
         cfg["l2"] = ("inputs+outputs of a step exceed the 126 MB L2; no explicit flush" if head["input_sets"] == 1 else
                      "launches rotate over %d input/output sets so that a launch does not find its operands in L2" % head["input_sets"])
         line = {
-            "metric": GEMM_METRIC if is_gemm else METRIC, "value": ctx.world * flops / (ms_per_step * 1e-3) / 1e12,
+            "metric": GEMM_METRIC if is_gemm else MOE_METRIC if is_moe else METRIC,
+            "value": ctx.world * flops / (ms_per_step * 1e-3) / 1e12,
             "unit": UNIT, "n_gpus": ctx.world, "steps": steps, "warmup": warmup, "ms_per_step": ms_per_step,
-            "higher_is_better": True, "scaling": args.scaling, "vs_baseline": None, "dtype": "bf16",
+            "higher_is_better": True, "scaling": args.scaling, "vs_baseline": None, "dtype": "fp8_e4m3" if is_moe else "bf16",
             "data": "synthetic", "config": cfg, "clocks": head["clocks"], "gpu_launches": head["gpu_launches"],
             "roofline": roofline, "input_sha256": head["input_sha256"],
         }

@@ -29,7 +29,7 @@ def test_default_headline_is_the_largest_prefill_configuration():
     args = bench.parse_args([])
     assert args.workload == "c4_long_context" and args.gpus == 1 and args.warmup >= 3
     for name in bench.PER_WORKLOAD_DEFAULT:
-        assert name.startswith("gemm_n") or name in inputs.WORKLOADS
+        assert name.startswith("gemm_n") or name in inputs.WORKLOADS or name in inputs.MOE_WORKLOADS
     for n in ("c1_tiny", "c2_mha_prefill", "c3_gqa_prefill", "c4_long_context", "c5_wide_noncausal",
               "paper_gqa_n1024", "paper_gqa_n16384"):
         assert n in bench.PER_WORKLOAD_DEFAULT
