@@ -34,6 +34,9 @@ ATTN_REGS_NEEDED = 128 * 64 + 256 * 216
 # The single-sub-tile kernel (OneCfg in csrc/attn_fwd_1t.cuh): 256 threads, 48 and 208 registers.
 ONE_THREADS = 256
 ONE_REGS_NEEDED = 128 * 48 + 128 * 208
+# The MoE GEMM (MoeGemmCfg in csrc/moe_fp8.cuh): 384 threads, 40 and 232 registers.
+MOE_THREADS = 384
+MOE_REGS_NEEDED = 128 * 40 + 256 * 232
 
 
 def _sources():
@@ -59,11 +62,12 @@ def kernel_registers(ptxas_report: str) -> dict:
 
 def check_register_split(ptxas_report: str) -> dict:
     """Raise if an attention kernel of the report cannot satisfy its register split."""
-    regs = {k: v for k, v in kernel_registers(ptxas_report).items() if "attn_fwd" in k}
+    regs = {k: v for k, v in kernel_registers(ptxas_report).items() if "attn_fwd" in k or "moe_gemm" in k}
     if not regs:
         raise RuntimeError("ptxas reported no attention kernel: cannot verify the register split")
     for name, n in regs.items():
-        threads, needed = (ONE_THREADS, ONE_REGS_NEEDED) if "attn_fwd_1t" in name else (ATTN_THREADS, ATTN_REGS_NEEDED)
+        threads, needed = (ONE_THREADS, ONE_REGS_NEEDED) if "attn_fwd_1t" in name else \
+            (MOE_THREADS, MOE_REGS_NEEDED) if "moe_gemm" in name else (ATTN_THREADS, ATTN_REGS_NEEDED)
         if threads * n < needed:
             raise RuntimeError("%s was compiled with %d registers per thread; its warp roles need %d x %d >= %d" % (
                 name, n, threads, n, needed))

@@ -202,11 +202,16 @@ bool register_split_fits_one_subtile(int regs_per_thread_at_launch) {
     return 128 * Cfg::kRegsLight + 128 * Cfg::kRegsSoftmax <= Cfg::kThreads * regs_per_thread_at_launch;
 }
 
+bool register_split_fits_moe_gemm(int regs_per_thread_at_launch) {
+    using Cfg = ave::MoeGemmCfg;
+    return 128 * Cfg::kRegsLight + 256 * Cfg::kRegsEpilogue <= Cfg::kThreads * regs_per_thread_at_launch;
+}
+
 // Which attention kernel ordinary (not split-KV) launches use: 0 = chosen per problem, 1 = always the
 // two-sub-tile kernel, 2 = always the single-sub-tile kernel (ave_attn_select_kernel).
 std::atomic<int> g_kernel_choice{0};
 
-// check_register_split: 0 = none, 1 = the two-sub-tile kernel's split, 2 = the single-sub-tile kernel's
+// check_register_split: 0 = none, 1 = the two-sub-tile kernel's split, 2 = the single-sub-tile kernel's, 3 = the MoE GEMM's
 template <class Kernel>
 int prepare_kernel(Kernel kern, int smem_bytes, int check_register_split, PerDeviceOnce &once) {
     int dev = -1;
@@ -215,8 +220,9 @@ int prepare_kernel(Kernel kern, int smem_bytes, int check_register_split, PerDev
     if (e == cudaSuccess && check_register_split) {
         cudaFuncAttributes attr;
         e = cudaFuncGetAttributes(&attr, kern);
-        if (e == cudaSuccess && !(check_register_split == 1 ? register_split_fits(attr.numRegs)
-                                                            : register_split_fits_one_subtile(attr.numRegs)))
+        if (e == cudaSuccess && !(check_register_split == 1   ? register_split_fits(attr.numRegs)
+                                  : check_register_split == 2 ? register_split_fits_one_subtile(attr.numRegs)
+                                                              : register_split_fits_moe_gemm(attr.numRegs)))
             return AVE_ERR_KERNEL_IMAGE;
     }
     // two CTAs of the single-sub-tile kernel share an SM: ask for the largest shared-memory carve-out
@@ -510,9 +516,9 @@ int launch_gemm(const void *a, const void *b, void *c, int M, int N, int K, cuda
     return launch_gemm_tile<256, B_NMAJOR>(a, b, c, M, N, K, sms, s);
 }
 
-// E4M3 codes [d3, d2, rows, inner] (inner contiguous) as a 4-D map with boxes of 128 bytes x 128 rows, 128-byte
-// swizzle.  (Not cached: two encodes per GEMM of a layer call.)
-bool encode_map_u8(CUtensorMap *map, const void *base, long long inner, long long rows, long long d2) {
+// E4M3 codes [d2, rows, inner] (inner contiguous) as a 4-D map with boxes of 128 bytes x box_rows rows, 128-byte
+// swizzle, zero fill outside.  (Not cached: two encodes per GEMM of a layer call.)
+bool encode_map_u8(CUtensorMap *map, const void *base, long long inner, long long rows, long long d2, int box_rows) {
     if (take_injected(g_inject_encode_failures)) {
         t_last_cuda_error = int(CUDA_ERROR_INVALID_VALUE);
         return false;
@@ -521,9 +527,32 @@ bool encode_map_u8(CUtensorMap *map, const void *base, long long inner, long lon
     if (!enc) return false;
     cuuint64_t gdim[4] = {cuuint64_t(inner), cuuint64_t(rows), cuuint64_t(d2), 1};
     cuuint64_t gstride[3] = {cuuint64_t(inner), cuuint64_t(inner) * cuuint64_t(rows), cuuint64_t(inner) * cuuint64_t(rows) * cuuint64_t(d2)};
-    cuuint32_t box[4] = {128, 128, 1, 1};
+    cuuint32_t box[4] = {128, cuuint32_t(box_rows), 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(base), gdim, gstride, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    g_map_encodes.fetch_add(1, std::memory_order_relaxed);
+    if (r != CUDA_SUCCESS) {
+        t_last_cuda_error = int(r);
+        return false;
+    }
+    return true;
+}
+
+// fp32 matrix [rows, cols] as a 4-D map {cols, rows, 1, 1} with boxes of 32 columns x 32 rows, 128-byte swizzle.
+bool encode_map_f32(CUtensorMap *map, const void *base, long long cols, long long rows) {
+    if (take_injected(g_inject_encode_failures)) {
+        t_last_cuda_error = int(CUDA_ERROR_INVALID_VALUE);
+        return false;
+    }
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return false;
+    cuuint64_t gdim[4] = {cuuint64_t(cols), cuuint64_t(rows), 1, 1};
+    cuuint64_t gstride[3] = {cuuint64_t(cols) * 4, cuuint64_t(cols) * cuuint64_t(rows) * 4, cuuint64_t(cols) * cuuint64_t(rows) * 4};
+    cuuint32_t box[4] = {32, 32, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void *>(base), gdim, gstride, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     g_map_encodes.fetch_add(1, std::memory_order_relaxed);
@@ -572,9 +601,10 @@ bool moe_layout(MoeWorkspace &w, int T, int C, int F, int E, int K) {
 int launch_moe_gemm(const void *a, long long rows, const float *a_scale, const void *b, const float *b_scale, int E,
                     int N, int K, const int *tile_expert, const float *row_weight, float *out, int sms, cudaStream_t s) {
     using Cfg = ave::MoeGemmCfg;
-    CUtensorMap ta, tb;
-    if (!encode_map_u8(&ta, a, K, rows, 1)) return AVE_ERR_CUDA;
-    if (!encode_map_u8(&tb, b, K, N, E)) return AVE_ERR_CUDA;
+    CUtensorMap ta, tb, tc;
+    if (!encode_map_u8(&ta, a, K, rows, 1, Cfg::kTile)) return AVE_ERR_CUDA;
+    if (!encode_map_u8(&tb, b, K, N, E, Cfg::kTileN)) return AVE_ERR_CUDA;
+    if (!encode_map_f32(&tc, out, N, rows)) return AVE_ERR_CUDA;
     ave::MoeGemmParams p;
     p.a_scale = a_scale;
     p.b_scale = b_scale;
@@ -582,11 +612,12 @@ int launch_moe_gemm(const void *a, long long rows, const float *a_scale, const v
     p.row_weight = row_weight;
     p.out = out;
     p.tiles_m = int(rows / 128);
-    p.tiles_n = N / 128;
+    p.tiles_n = (N + Cfg::kTileN - 1) / Cfg::kTileN;
+    p.nblk = N / 128;
     p.kb = K / 128;
     p.N = N;
     static PerDeviceOnce once;
-    const int st = prepare_kernel(ave::moe_gemm_fp8_kernel, Cfg::kSmemBytes, 0, once);
+    const int st = prepare_kernel(ave::moe_gemm_fp8_kernel, Cfg::kSmemBytes, 3, once);
     if (st != AVE_OK) return st;
     if (take_injected(g_inject_launch_failures)) {
         t_last_cuda_error = int(cudaErrorLaunchFailure);
@@ -594,7 +625,7 @@ int launch_moe_gemm(const void *a, long long rows, const float *a_scale, const v
     }
     const long long n_tiles = (long long)p.tiles_m * p.tiles_n;
     const unsigned grid = unsigned(n_tiles < sms ? n_tiles : sms);
-    ave::moe_gemm_fp8_kernel<<<dim3(grid), dim3(Cfg::kThreads), Cfg::kSmemBytes, s>>>(ta, tb, p);
+    ave::moe_gemm_fp8_kernel<<<dim3(grid), dim3(Cfg::kThreads), Cfg::kSmemBytes, s>>>(ta, tb, tc, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
         t_last_cuda_error = int(e);

@@ -12,17 +12,17 @@
 //   5. moe_gemm_fp8_kernel: o = w * (a W2^T), rows x C, fp32   (w: the pair's routing weight)
 //   6. moe_combine_kernel: y[t] = sum over the token's K rows of o, rounded to bf16
 //
-// The GEMM: persistent CTAs over 128 x 128 output tiles; K is streamed in blocks of 128 (one scale block)
-// through a TMA ring; each block is four M128 x N128 x K32 tcgen05 MMAs (kind::f8f6f4) into one of four TMEM
-// accumulators, which the epilogue warps read out and add, multiplied by the block's two scales, to fp32
+// The GEMM: persistent CTAs over 128 x 256 output tiles; K is streamed in blocks of 128 (one scale block)
+// through a TMA ring; each block is four M128 x N256 x K32 tcgen05 MMAs (kind::f8f6f4) into one of two TMEM
+// accumulators, which the epilogue warps read out and add, multiplied by the block's scales, to fp32
 // registers (the accumulation across scale blocks cannot stay in the tensor core: every block has its own
-// factor).  Rows are TMEM lanes, one epilogue thread per row.
+// factor).  Rows are TMEM lanes; two epilogue threads per row, 128 columns (one weight scale block) each.
 //
-//   warp 0      producer: TMA loads of the A and B blocks
-//   warp 1      MMA issuer
-//   warp 2      TMEM allocation / release
-//   warp 3      -
-//   warps 4..7  epilogue (thread = output row)
+//   warp 0       producer: TMA loads of the A and B blocks
+//   warp 1       MMA issuer
+//   warp 2       TMEM allocation / release
+//   warp 3       -
+//   warps 4..11  epilogue (thread = output row x half of the tile's columns)
 #pragma once
 
 #include <cuda_bf16.h>
@@ -34,14 +34,22 @@ namespace ave {
 constexpr int kMoeGroup = 128;  // channels per activation scale, rows and columns per weight scale block
 
 struct MoeGemmCfg {
-    static constexpr int kThreads = 256;
-    static constexpr int kTile = 128;                          // output tile 128 x 128, K block 128
-    static constexpr int kStages = 6;
+    static constexpr int kThreads = 384;
+    static constexpr int kTile = 128;                          // rows of an output tile; K block; columns per epilogue thread
+    static constexpr int kTileN = 256;                         // columns of an output tile
+    static constexpr int kStages = 4;
     static constexpr int kABytes = kTile * kMoeGroup;          // 16 KB of E4M3
-    static constexpr int kStageBytes = 2 * kABytes;
-    static constexpr int kSmemBytes = kStages * kStageBytes + 1024;
-    static constexpr int kAccs = 4;                            // TMEM accumulators of 128 columns
-    static constexpr uint32_t kTmemCols = kAccs * kTile;
+    static constexpr int kBBytes = kTileN * kMoeGroup;         // 32 KB
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kStageCBytes = 8 * 32 * 128;          // result staging: 32 rows x 32 fp32 per epilogue warp
+    static constexpr int kSmemBytes = kStages * kStageBytes + kStageCBytes + 1024;
+    static constexpr int kAccs = 2;                            // TMEM accumulators of 256 columns
+    static constexpr uint32_t kTmemCols = kAccs * kTileN;
+    // The epilogue threads hold 128 fp32 sums plus two 32-column chunks in flight: they take registers from the
+    // producer / MMA warpgroup (setmaxnreg moves them inside the CTA's allocation of kThreads x kRegsAtLaunch;
+    // the build and the launch code check the compiled image against this split).
+    static constexpr int kRegsLight = 40, kRegsEpilogue = 232, kRegsAtLaunch = 168;
+    static_assert(128 * kRegsLight + 256 * kRegsEpilogue <= kThreads * kRegsAtLaunch, "register split exceeds the CTA's allocation");
 };
 
 struct MoeGemmParams {
@@ -50,7 +58,8 @@ struct MoeGemmParams {
     const int *tile_expert;   // [rows/128]: expert of each 128-row tile of the sorted order, -1 = unused tile
     const float *row_weight;  // [rows] or NULL: factor applied to every output row
     float *out;               // [rows, N] fp32
-    int tiles_m, tiles_n;     // rows / 128, N / 128
+    int tiles_m, tiles_n;     // rows / 128, ceil(N / 256)
+    int nblk;                 // N / 128: weight scale blocks along N
     int kb;                   // K / 128
     int N;
 };
@@ -92,10 +101,13 @@ __device__ __forceinline__ void moe_tile_coords(int id, const MoeGemmParams &p, 
     bm = m0 + (rem - bn * gm);
 }
 
-// tm_a: A codes [rows, K] as {K, rows, 1, 1}; tm_b: B codes [E, N, K] as {K, N, E, 1}; boxes of 128 x 128 bytes.
-__global__ void __launch_bounds__(256, 1)
+// tm_a: A codes [rows, K] as {K, rows, 1, 1}, boxes of 128 bytes x 128 rows; tm_b: B codes [E, N, K] as
+// {K, N, E, 1}, boxes of 128 bytes x 256 rows (rows beyond N read as zero); tm_c: the fp32 result [rows, N] as
+// {N, rows, 1, 1}, boxes of 32 columns x 32 rows (a thread-per-row store of fp32 rows would touch 32 rows per
+// instruction, one sector each: measured, that cost more than the tile's products).
+__global__ void __launch_bounds__(384, 1)
 moe_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                    const MoeGemmParams p) {
+                    const __grid_constant__ CUtensorMap tm_c, const MoeGemmParams p) {
     using Cfg = MoeGemmCfg;
     constexpr int NS = Cfg::kStages, NA = Cfg::kAccs;
     extern __shared__ uint8_t smem_raw[];
@@ -116,7 +128,7 @@ moe_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         }
         for (int a = 0; a < NA; ++a) {
             mbar_init(smem_u32(&bar_acc_full[a]), 1);
-            mbar_init(smem_u32(&bar_acc_empty[a]), 4);  // one arrival per epilogue warp
+            mbar_init(smem_u32(&bar_acc_empty[a]), 8);  // one arrival per epilogue warp
         }
         mbar_init(smem_u32(&bar_drain), 1);
         fence_mbar_init();
@@ -140,7 +152,9 @@ moe_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
 
     if (poisoned) {
         // nothing: fall through to the common exit
-    } else if (warp == 0) {
+    } else if (warp < 4) {
+      setmaxnreg_dec<Cfg::kRegsLight>();
+      if (warp == 0) {
         // =============================== producer ===============================
         const bool leader = elect_one();
         if (leader) {
@@ -165,7 +179,7 @@ moe_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                     const uint32_t dst = sRing + slot * Cfg::kStageBytes;
                     mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
                     tma_load_4d(dst, &tm_a, bar, kb * kMoeGroup, bm * Cfg::kTile, 0, 0);
-                    tma_load_4d(dst + Cfg::kABytes, &tm_b, bar, kb * kMoeGroup, bn * Cfg::kTile, e, 0);
+                    tma_load_4d(dst + Cfg::kABytes, &tm_b, bar, kb * kMoeGroup, bn * Cfg::kTileN, e, 0);
                 }
             }
         }
@@ -176,7 +190,7 @@ moe_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     } else if (warp == 1) {
         // =============================== MMA issuer ===============================
         const bool leader = elect_one();
-        constexpr uint32_t idesc = make_idesc_e4m3(Cfg::kTile, Cfg::kTile);
+        constexpr uint32_t idesc = make_idesc_e4m3(Cfg::kTile, Cfg::kTileN);
         constexpr uint64_t desc_kmajor = make_sdesc_sw128(16, 1024);  // rows of 128 bytes, 8-row atoms of 1024 bytes
         constexpr uint32_t hi = uint32_t(desc_kmajor >> 32), lo = uint32_t(desc_kmajor);
         bool ok = true;
@@ -197,7 +211,7 @@ moe_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                 if (leader) {
                     const uint32_t a_lo = lo | ((sRing + slot * Cfg::kStageBytes) >> 4);
                     const uint32_t b_lo = lo | ((sRing + slot * Cfg::kStageBytes + Cfg::kABytes) >> 4);
-                    const uint32_t d_tmem = tmem + acc * Cfg::kTile;
+                    const uint32_t d_tmem = tmem + acc * Cfg::kTileN;
 #pragma unroll
                     for (int kk = 0; kk < kMoeGroup / 32; ++kk)  // K = 32 bytes per instruction
                         umma_f8_ss_words(d_tmem, a_lo + ((kk * 32) >> 4), hi, b_lo + ((kk * 32) >> 4), hi, idesc, kk > 0);
@@ -210,10 +224,15 @@ moe_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             if (leader) umma_commit(smem_u32(&bar_drain));
             for (uint32_t w = 0; w < WAIT_LIMIT && !mbar_test_wait(smem_u32(&bar_drain), 0); ++w) {}
         }
-    } else if (warp >= 4) {
+      }
+    } else {
         // =============================== epilogue ===============================
-        const int wq = warp & 3;  // TMEM lane quadrant of this warp
+        setmaxnreg_inc<Cfg::kRegsEpilogue>();
+        const int wq = warp & 3;           // TMEM lane quadrant of this warp
+        const int half = (warp - 4) >> 2;  // which 128 of the tile's 256 columns
         const uint32_t lane_sel = uint32_t(wq * 32) << 16;
+        const uint32_t sC = sRing + NS * Cfg::kStageBytes + (warp - 4) * (32 * 128);  // this warp's 32 staging rows
+        bool store_pending = false;  // (lane 0) a TMA store may still be reading the staging rows
         bool ok = true;
         int ring = 0;
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
@@ -222,8 +241,10 @@ moe_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             const int e = p.tile_expert[bm];
             if (e < 0) continue;
             const int row = bm * Cfg::kTile + wq * 32 + lane;
+            const int nb = bn * 2 + half;              // this thread's weight scale block along N
+            const bool live = nb < p.nblk;             // (the last tile's second half lies beyond N when N % 256 == 128)
             const float *sa = p.a_scale + size_t(row) * p.kb;
-            const float *sb = p.b_scale + (size_t(e) * p.tiles_n + bn) * p.kb;
+            const float *sb = p.b_scale + (size_t(e) * p.nblk + (live ? nb : 0)) * p.kb;
             float acc[Cfg::kTile];
 #pragma unroll
             for (int c = 0; c < Cfg::kTile; ++c) acc[c] = 0.f;
@@ -235,28 +256,52 @@ moe_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                 ok = wait_bar(&bar_acc_full[a], (ring / NA) & 1, STATUS_TIMEOUT_MMA);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t t_acc = tmem + a * Cfg::kTile + lane_sel;
+                const uint32_t t_acc = tmem + a * Cfg::kTileN + half * Cfg::kTile + lane_sel;
+                // 32 columns at a time, the next chunk's load in flight while this chunk is added up
+                uint32_t v[2][32];
+                tmem_ld_x32(t_acc, v[0]);
 #pragma unroll
                 for (int c = 0; c < Cfg::kTile / 32; ++c) {
-                    uint32_t v[32];
-                    tmem_ld_x32(t_acc + c * 32, v);
                     tmem_wait_ld();
-                    if (c == Cfg::kTile / 32 - 1) {  // the block's products are in registers: the accumulator is free
+                    if (c + 1 < Cfg::kTile / 32) {
+                        tmem_ld_x32(t_acc + (c + 1) * 32, v[(c + 1) & 1]);
+                    } else {  // the block's products are in registers: the accumulator is free
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[a]));
                     }
 #pragma unroll
-                    for (int x = 0; x < 32; ++x) acc[c * 32 + x] = fmaf(__uint_as_float(v[x]), s, acc[c * 32 + x]);
+                    for (int x = 0; x < 32; ++x) acc[c * 32 + x] = fmaf(__uint_as_float(v[c & 1][x]), s, acc[c * 32 + x]);
                 }
             }
             if (!ok) break;
+            if (!live) continue;
             const float w = p.row_weight ? p.row_weight[row] : 1.f;
-            float4 *dst = reinterpret_cast<float4 *>(p.out + size_t(row) * p.N + size_t(bn) * Cfg::kTile);
+            // 32 columns at a time through this warp's staging rows (128 bytes each, 128-byte swizzle) and out by TMA
 #pragma unroll
-            for (int c = 0; c < Cfg::kTile; c += 4)
-                dst[c >> 2] = make_float4(acc[c] * w, acc[c + 1] * w, acc[c + 2] * w, acc[c + 3] * w);
+            for (int c = 0; c < Cfg::kTile / 32; ++c) {
+                if (store_pending) {
+                    if (lane == 0) tma_store_wait_read();
+                    __syncwarp();
+                }
+#pragma unroll
+                for (int x = 0; x < 32; x += 4) {
+                    const uint32_t addr = sC + lane * 128 + ((uint32_t(x >> 2) ^ uint32_t(lane & 7)) << 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr),
+                                 "r"(__float_as_uint(acc[c * 32 + x] * w)), "r"(__float_as_uint(acc[c * 32 + x + 1] * w)),
+                                 "r"(__float_as_uint(acc[c * 32 + x + 2] * w)), "r"(__float_as_uint(acc[c * 32 + x + 3] * w))
+                                 : "memory");
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_4d(&tm_c, sC, nb * Cfg::kTile + c * 32, bm * Cfg::kTile + wq * 32, 0, 0);
+                    tma_store_commit();
+                }
+                store_pending = true;
+            }
         }
+        if (lane == 0 && store_pending) tma_store_wait_all();
     }
 
     // ---- common exit: every thread arrives, then TMEM is released
