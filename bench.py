@@ -53,7 +53,7 @@ PER_WORKLOAD_DEFAULT = [
     "d192_gqa_prefill", "d256_gqa_prefill",
     "decode_mha_b8_k8192", "decode_gqa_b8_k16384", "decode_gqa_b1_k65536", "decode_gqa_b64_k4096",
     "gemm_n4096", "gemm_n8192", "gemm_n16384",
-    "moe_t1024", "moe_t4096", "moe_t16384",
+    "moe_t4096", "moe_t16384",
 ]
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel, from profiler captures of the
 # kernel as committed; a workload whose kernel has changed since its capture is absent (reported as null).

@@ -193,26 +193,59 @@ MOE_WORKLOADS = {n: MoeWorkload(n, t, seed=400 + i) for i, (n, t) in enumerate(
     (("moe_t256", 256), ("moe_t1024", 1024), ("moe_t4096", 4096), ("moe_t8192", 8192), ("moe_t16384", 16384)))}
 
 
+# Exponent field of a random E4M3 code, looked up with a uniform byte: most values within a factor of 8 below the
+# block maximum, as in block-quantised Gaussian data.  (A table of bit patterns; nothing here evaluates the format.)
+_EXPO_OF_BYTE = torch.tensor([15] * 26 + [14] * 82 + [13] * 72 + [12] * 38 + [11] * 20 + [10] * 10 + [9] * 5 + [8] * 3,
+                             dtype=torch.uint8)
+assert _EXPO_OF_BYTE.numel() == 256
+
+
 def _fp8_codes(g: torch.Generator, shape, group_axis_len: int):
-    """Random E4M3 bit patterns shaped like block-quantised Gaussian data: the exponent field is drawn from a
-    fixed table of weights (most values within a factor of 8 below the block maximum), mantissa and sign
-    uniformly; the first element of every group of 128 along the last axis is the block maximum (+-448, code
-    0x7e), as it is after scaling a block by its largest magnitude.  No NaN pattern is produced.  Bit patterns
-    only: nothing here evaluates the format."""
-    n = 1
-    for d in shape:
-        n *= d
-    weights = torch.zeros(16)
-    weights[15], weights[14], weights[13], weights[12], weights[11] = 0.10, 0.32, 0.28, 0.15, 0.08
-    weights[10], weights[9], weights[8] = 0.04, 0.02, 0.01
-    expo = torch.multinomial(weights, n, replacement=True, generator=g).to(torch.uint8)
-    mant = torch.randint(0, 8, (n,), generator=g, dtype=torch.uint8)
-    mant = torch.where((expo == 15) & (mant == 7), torch.zeros_like(mant), mant)   # 0x7f would be NaN
-    sign = torch.randint(0, 2, (n,), generator=g, dtype=torch.uint8) << 7
-    codes = (sign | (expo << 3) | mant).reshape(shape)
-    lead = codes[..., ::group_axis_len]
-    codes[..., ::group_axis_len] = (lead & 0x80) | 0x7E
-    return codes.contiguous()
+    """Random E4M3 bit patterns shaped like block-quantised Gaussian data: exponent field from the table above,
+    mantissa and sign uniform; the first element of every group of 128 along the last axis is the block maximum
+    (+-448, code 0x7e), as it is after scaling a block by its largest magnitude.  No NaN pattern is produced."""
+    out = torch.empty(shape, dtype=torch.uint8)
+    flat = out.view(-1)
+    n = flat.numel()
+    step = 1 << 26
+    for lo in range(0, n, step):
+        m = min(step, n - lo)
+        expo = _EXPO_OF_BYTE[torch.randint(0, 256, (m,), generator=g, dtype=torch.int64)]
+        low = torch.randint(0, 16, (m,), generator=g, dtype=torch.uint8)       # sign bit and mantissa
+        mant = low & 7
+        mant = torch.where((expo == 15) & (mant == 7), torch.zeros_like(mant), mant)   # 0x7f would be NaN
+        flat[lo:lo + m] = ((low >> 3) << 7) | (expo << 3) | mant
+    lead = out[..., ::group_axis_len]
+    out[..., ::group_axis_len] = (lead & 0x80) | 0x7E
+    return out
+
+
+def _expert_codes(g: torch.Generator, E: int, rows: int, cols: int):
+    """[E, rows, cols] codes: four experts are drawn; expert e repeats expert e % 4 rotated by 128 * (e // 4) columns
+    (drawing 1.4 G independent codes takes most of a minute; the experts' scales are all different)."""
+    base = _fp8_codes(g, (min(E, 4), rows, cols), 128)
+    out = torch.empty((E, rows, cols), dtype=torch.uint8)
+    for e in range(E):
+        out[e] = torch.roll(base[e % 4], shifts=128 * (e // 4), dims=1) if e >= 4 else base[e]
+    return out
+
+
+_MOE_WEIGHTS = {}
+
+
+def _moe_weights(C: int, F: int, E: int):
+    """The layer's quantised weights: one set per (C, F, E), shared by the workloads of every token count (seed 4000)."""
+    key = (C, F, E)
+    if key not in _MOE_WEIGHTS:
+        g = torch.Generator(device="cpu")
+        g.manual_seed(4000)
+        w13q = _expert_codes(g, E, 2 * F, C)
+        s13 = ((0.8 + 0.4 * torch.rand((E, 2 * F // 128, C // 128), generator=g)) * (2.8 / 448.0 / math.sqrt(C))).float()
+        w2q = _expert_codes(g, E, C, F)
+        s2 = ((0.8 + 0.4 * torch.rand((E, C // 128, F // 128), generator=g)) * (2.8 / 448.0 / math.sqrt(F))).float()
+        _MOE_WEIGHTS.clear()      # one set at a time: the paper's configuration is 1.4 GB
+        _MOE_WEIGHTS[key] = (w13q, s13, w2q, s2)
+    return _MOE_WEIGHTS[key]
 
 
 def make_moe_inputs(w: MoeWorkload):
@@ -224,15 +257,12 @@ def make_moe_inputs(w: MoeWorkload):
     g.manual_seed(w.seed)
     T, C, F, E, K = w.T, w.C, w.F, w.E, w.K
     xq = _fp8_codes(g, (T, C), 128)
-    sx = (0.8 + 0.4 * torch.rand((T, C // 128), generator=g)) * (2.8 / 448.0)
-    w13q = _fp8_codes(g, (E, 2 * F, C), 128)
-    s13 = (0.8 + 0.4 * torch.rand((E, 2 * F // 128, C // 128), generator=g)) * (2.8 / 448.0 / math.sqrt(C))
-    w2q = _fp8_codes(g, (E, C, F), 128)
-    s2 = (0.8 + 0.4 * torch.rand((E, C // 128, F // 128), generator=g)) * (2.8 / 448.0 / math.sqrt(F))
-    ids = torch.stack([torch.randperm(E, generator=g)[:K] for _ in range(T)]).to(torch.int32)
+    sx = ((0.8 + 0.4 * torch.rand((T, C // 128), generator=g)) * (2.8 / 448.0)).float()
+    w13q, s13, w2q, s2 = _moe_weights(C, F, E)
+    ids = torch.argsort(torch.rand((T, E), generator=g), dim=1)[:, :K].to(torch.int32).contiguous()
     raw = 0.1 + torch.rand((T, K), generator=g)
     wts = (raw / raw.sum(dim=1, keepdim=True)).to(torch.float32)
-    return xq, sx.float(), w13q, s13.float(), w2q, s2.float(), ids, wts
+    return xq, sx, w13q, s13, w2q, s2, ids, wts
 
 
 def moe_flops(w: MoeWorkload) -> float:
