@@ -389,8 +389,12 @@ attn_fwd_1t_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 float m_run = -INFINITY, l_run = 0.f;
                 const int k_end = key_end(w, p);
                 const int n_full = unmasked_steps<CAUSAL, SPLIT>(i0, n_t, key_begin(w), k_end, off, p.rows_per_head);
-                auto step = [&](const int j, auto masked_tag) -> bool {
-                    constexpr bool need_mask = decltype(masked_tag)::value;
+                auto step = [&](const int j, auto masked) -> bool {
+                    // `masked` is a run-time bool (causal kernels) or std::true_type / std::false_type
+                    constexpr bool kRuntimeFlag = std::is_same<decltype(masked), bool>::value;
+                    bool need_mask;
+                    if constexpr (kRuntimeFlag) need_mask = masked;
+                    else need_mask = decltype(masked)::value;
                     ok = wait_bar(&bar_s, ns & 1, STATUS_TIMEOUT_MMA);
                     if (!ok) return false;
                     ++ns;
@@ -399,7 +403,9 @@ attn_fwd_1t_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
                     for (int c = 0; c < 4; ++c) tmem_ld_x32(tS + c * 32, sraw[c]);
                     tmem_wait_ld();
-                    if (need_mask) {
+                    const int mask_trips = kRuntimeFlag ? opaque(need_mask ? 1 : 0) : int(need_mask);
+#pragma unroll 1
+                    for (int trip = 0; trip < mask_trips; ++trip) {
                         const int j0 = key_begin(w) + j * BN;  // first key of this step
                         int lim = k_end - 1 - j0;               // columns c <= lim of this tile are visible to row i
                         if constexpr (SPLIT) {
@@ -482,11 +488,17 @@ attn_fwd_1t_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     return true;
                 };
                 {
-                    int j = 0;
-                    for (; j < n_full; ++j)
-                        if (!step(j, std::false_type{})) break;
-                    for (; ok && j < n_t; ++j)
-                        if (!step(j, std::true_type{})) break;
+                    if constexpr (CAUSAL) {
+                        for (int j = 0; j < n_t; ++j)
+                            if (!step(j, j >= n_full)) break;
+                    } else {
+                        // only a ragged last key tile is masked here: a copy of the step for it costs nothing
+                        int j = 0;
+                        for (; j < n_full; ++j)
+                            if (!step(j, std::false_type{})) break;
+                        for (; ok && j < n_t; ++j)
+                            if (!step(j, std::true_type{})) break;
+                    }
                 }
 
                 // ---- epilogue: O / l -> bf16 -> global (each thread its own row); LSE = ln2 * (m + log2 l)

@@ -522,13 +522,18 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             } else {
                 float m_run = -INFINITY, l_run = 0.f;
                 // Steps [0, n_full) lie wholly below the causal diagonal and inside the key range: nothing
-                // to mask.  The step is instantiated twice, with and without the masking code, and the
-                // choice is made once per tile here: left as a run-time flag inside one body, the
-                // per-element compares and selects end up predicated into every step.
+                // to mask.  In the causal kernels the masking code sits in a loop of zero or one trips whose
+                // count the compiler cannot see: a plain `if` ends up predicated into every step, and a
+                // second copy of the step for the masked case is cold in the instruction cache at every
+                // tile's diagonal (a masked step then took three times as long as an unmasked one).
                 const int k_end = key_end(w, p);
                 const int n_full = unmasked_steps<CAUSAL, SPLIT>(i0, n_t, key_begin(w), k_end, off, p.rows_per_head);
-                auto step = [&](const int j, auto masked_tag) -> bool {
-                    constexpr bool need_mask = decltype(masked_tag)::value;
+                auto step = [&](const int j, auto masked) -> bool {
+                    // `masked` is a run-time bool (causal kernels) or std::true_type / std::false_type
+                    constexpr bool kRuntimeFlag = std::is_same<decltype(masked), bool>::value;
+                    bool need_mask;
+                    if constexpr (kRuntimeFlag) need_mask = masked;
+                    else need_mask = decltype(masked)::value;
                     if (traced(n) && tracer) trace_stamp(1 + t, trace_it(n, j), 0);
                     ok = wait_bar(&bar_s[t], ns & 1, STATUS_TIMEOUT_MMA);
                     if (!ok) return false;
@@ -552,7 +557,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 
                     // ---- row maximum of the raw scores.  A masked score is simply replaced by -inf: it then
                     // drops out of the maximum and its probability exp2(-inf) is exactly 0.
-                    if (need_mask) {
+                    const int mask_trips = kRuntimeFlag ? opaque(need_mask ? 1 : 0) : int(need_mask);
+#pragma unroll 1
+                    for (int trip = 0; trip < mask_trips; ++trip) {
 #pragma unroll
                         for (int c = 0; c < 128; ++c)
                             sraw[c >> 5][c & 31] = (c <= lim) ? sraw[c >> 5][c & 31] : 0xff800000u;
@@ -661,11 +668,17 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     return true;
                 };
                 {
-                    int j = 0;
-                    for (; j < n_full; ++j)
-                        if (!step(j, std::false_type{})) break;
-                    for (; ok && j < n_t; ++j)
-                        if (!step(j, std::true_type{})) break;
+                    if constexpr (CAUSAL) {
+                        for (int j = 0; j < n_t; ++j)
+                            if (!step(j, j >= n_full)) break;
+                    } else {
+                        // only a ragged last key tile is masked here: a copy of the step for it costs nothing
+                        int j = 0;
+                        for (; j < n_full; ++j)
+                            if (!step(j, std::false_type{})) break;
+                        for (; ok && j < n_t; ++j)
+                            if (!step(j, std::true_type{})) break;
+                    }
                 }
 
                 // ---- epilogue: O / l -> bf16 -> shared (TMA layout) -> global; LSE = ln2 * (m + log2 l)

@@ -10,6 +10,15 @@
 
 namespace ave {
 
+// Returns x through an empty asm statement, so that the compiler knows nothing about the value.  Used
+// for the trip count (0 or 1) of a loop around code that only a few steps need: as a plain `if`, the
+// compiler predicates such a block into every step; as a second instantiation of the step, the copy is
+// tens of KB of instructions that are cold in the instruction cache whenever a tile reaches them.
+__device__ __forceinline__ int opaque(int x) {
+    asm volatile("" : "+r"(x));
+    return x;
+}
+
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float r;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
