@@ -58,8 +58,18 @@ __device__ long long g_trace[TRACE_ROLES][TRACE_ITERS][TRACE_SLOTS];
 __device__ __forceinline__ void trace_stamp(int role, int iter, int slot) {
     if (blockIdx.x == AVE_TRACE && iter < TRACE_ITERS) g_trace[role][iter][slot] = clock64();
 }
+// Life span of every CTA of the last launch: global-timer nanoseconds at its first and last instruction
+// and the number of work tiles it processed (how long the grid takes to start, how ragged its end is).
+constexpr int TRACE_CTAS = 8192;
+__device__ unsigned long long g_cta_span[TRACE_CTAS][3];
+__device__ __forceinline__ void span_stamp(int slot, unsigned long long value = ~0ull) {
+    if (blockIdx.x >= TRACE_CTAS) return;
+    if (value == ~0ull) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(value));
+    g_cta_span[blockIdx.x][slot] = value;
+}
 #else
 __device__ __forceinline__ void trace_stamp(int, int, int) {}
+__device__ __forceinline__ void span_stamp(int, unsigned long long = 0) {}
 #endif
 
 // Wait for an mbarrier phase, for a bounded TIME (one mbarrier.try_wait may

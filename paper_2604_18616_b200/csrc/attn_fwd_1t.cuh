@@ -61,6 +61,7 @@ template <int D, bool CAUSAL, bool SPLIT, bool VARLEN = false>
 __global__ void __launch_bounds__(256, 2)
 attn_fwd_1t_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v, const FwdParams p) {
+    if (threadIdx.x == 0) span_stamp(0);
     using Cfg = OneCfg<D>;
     using Tile = TileOf<SPLIT, VARLEN>;
     constexpr int NS = Cfg::kStages;
@@ -138,10 +139,16 @@ attn_fwd_1t_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             // =============================== tile scheduler ===============================
             const bool leader = elect_one();
             bool ok = true;
+            int last_id = blockIdx.x;   // the newest tile this CTA holds
             for (int k = 0; ok; ++k) {
                 const int slot = k & 1;
                 if (k >= 2) {  // every consumer has read the tile this slot held two requests ago
                     ok = wait_bar(&bar_tile_empty[slot], ((k >> 1) - 1) & 1, STATUS_TIMEOUT_SLOT);
+                    if (!ok) break;
+                }
+                // over the launch's last tiles requests run one tile ahead, not two (see the two-sub-tile kernel)
+                if (k >= 1 && p.total_blocks - last_id <= kLastWaves * Cfg::kCtasPerSm * int(n_sm())) {
+                    ok = wait_bar(&bar_tile_empty[slot ^ 1], ((k - 1) >> 1) & 1, STATUS_TIMEOUT_SLOT);
                     if (!ok) break;
                 }
                 if (leader) {
@@ -160,6 +167,7 @@ attn_fwd_1t_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bar_tile_ready[slot]));
                 if (id < 0) break;  // nothing left to take over: never ask again
+                last_id = id;
             }
         } else if (warp == 0) {
             // =============================== producer ===============================
@@ -557,6 +565,7 @@ attn_fwd_1t_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     tc_fence_before();
     __syncthreads();
     if (warp == 2) tmem_dealloc(tmem, Cfg::kTmemCols);
+    if (threadIdx.x == 0) span_stamp(1);
 }
 
 }  // namespace ave

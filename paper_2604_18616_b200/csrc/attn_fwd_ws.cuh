@@ -54,6 +54,9 @@ struct WsCfg {
     static constexpr int kTileConsumers = 10;               // producer + MMA + 8 softmax warps read each tile id
 };
 
+// Over the last kLastWaves x (resident CTAs) tiles of a launch a CTA claims one tile ahead instead of two.
+constexpr int kLastWaves = 2;
+
 // Rescale O only when the running maximum moved by more than this many powers of two; until then
 // probabilities are taken relative to a stale maximum (at most 2^32 too large), which the final division by l
 // undoes.  Nothing is lost by a large threshold: P is rounded to bf16, which has fp32's exponent range, and
@@ -117,6 +120,7 @@ __global__ void __launch_bounds__(384, 1)
 attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
                    const FwdParams p) {
+    if (threadIdx.x == 0) span_stamp(0);
     using Cfg = WsCfg<D>;
     constexpr int NS = Cfg::kStages;
     extern __shared__ uint8_t smem_raw[];
@@ -198,10 +202,21 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             // =============================== tile scheduler ===============================
             const bool leader = elect_one();
             bool ok = true;
+            int last_id = blockIdx.x;   // the newest tile this CTA holds
             for (int k = 0; ok; ++k) {
                 const int slot = k & 1;
                 if (k >= 2) {  // every consumer has read the response this slot held two requests ago
                     ok = wait_bar(&bar_tile_empty[slot], ((k >> 1) - 1) & 1, STATUS_TIMEOUT_SLOT);
+                    if (!ok) break;
+                }
+                // Requests normally run two tiles ahead of the tile the CTA works on.  Over the launch's last
+                // tiles they run one ahead only (request k waits until every warp has read response k-1,
+                // that is, has begun the tile it named): a tile claimed early there is one that an SM about
+                // to go idle could have taken.  With two ahead throughout, the last CTA of a 2048-token
+                // causal launch ended 30 us after the median one; with one ahead throughout, the MMA warp
+                // waits for its next tile at many tile ends.
+                if (k >= 1 && p.total_blocks - last_id <= kLastWaves * int(n_sm())) {
+                    ok = wait_bar(&bar_tile_empty[slot ^ 1], ((k - 1) >> 1) & 1, STATUS_TIMEOUT_SLOT);
                     if (!ok) break;
                 }
                 if (leader) {
@@ -220,6 +235,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bar_tile_ready[slot]));
                 if (id < 0) break;  // nothing left to take over: never ask again
+                last_id = id;
             }
         } else if (warp == 0) {
             // =============================== producer ===============================
@@ -460,6 +476,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 ring = ring_next;
                 id = id_next;
                 w = w_next;
+                if (lane == 0) span_stamp(2, n + 1);
             }
             if (!ok) {  // abandoned: let the MMAs already issued finish before TMEM is released
                 if (leader) umma_commit(smem_u32(&bar_drain));
@@ -771,6 +788,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     tc_fence_before();
     __syncthreads();
     if (warp == 2) tmem_dealloc(tmem, Cfg::kTmemCols);
+    if (threadIdx.x == 0) span_stamp(1);
 }
 
 }  // namespace ave

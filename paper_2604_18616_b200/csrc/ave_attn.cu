@@ -988,6 +988,19 @@ int ave_attn_trace_read(long long *out) {
     if (e == cudaSuccess) e = cudaMemcpyFromSymbol(out, ave::g_trace, sizeof(ave::g_trace));
     return e == cudaSuccess ? AVE_OK : AVE_ERR_CUDA;
 }
+// The life span of the last launch's CTAs: n_ctas x {first ns, last ns, tiles processed}.
+int ave_attn_trace_read_spans(unsigned long long *out, int n_ctas) {
+    if (n_ctas > ave::TRACE_CTAS) n_ctas = ave::TRACE_CTAS;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpyFromSymbol(out, ave::g_cta_span, size_t(n_ctas) * 3 * sizeof(unsigned long long));
+    return e == cudaSuccess ? AVE_OK : AVE_ERR_CUDA;
+}
+int ave_attn_trace_clear_spans() {
+    void *ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&ptr, ave::g_cta_span);
+    if (e == cudaSuccess) e = cudaMemset(ptr, 0, sizeof(ave::g_cta_span));
+    return e == cudaSuccess ? AVE_OK : AVE_ERR_CUDA;
+}
 #endif
 
 static int gemm_validate(const void *a, const void *b, const void *c, int M, int N, int K) {

@@ -129,6 +129,13 @@ __device__ __forceinline__ void tmem_wait_st() {
 }
 
 // ------------------------------------------------------------------------ MMA
+// Number of SMs of the device.
+__device__ __forceinline__ uint32_t n_sm() {
+    uint32_t n;
+    asm("mov.u32 %0, %%nsmid;" : "=r"(n));
+    return n;
+}
+
 // D[tmem] (+)= A[smem] * B[smem], and D[tmem] (+)= A[tmem] * B[smem]; each issued by ONE thread.
 // A 64-bit shared-memory descriptor is given as its (low, high) 32-bit words.
 __device__ __forceinline__ void umma_ss_words(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,

@@ -69,11 +69,35 @@ def events(stamps):
     return out
 
 
+def span_summary(spans, sms=148):
+    """Text summary of per-CTA (first ns, last ns, tiles) triples of one launch; CTAs that never ran
+    (their index was taken over by a running CTA) have a zero start."""
+    ran = [(a, b, t) for a, b, t in spans if a > 0 and b >= a]
+    if not ran:
+        return "no CTA ran"
+    t0 = min(a for a, _, _ in ran)
+    t1 = max(b for _, b, _ in ran)
+    starts = sorted(a - t0 for a, _, _ in ran)
+    ends = sorted(t1 - b for _, b, _ in ran)
+    busy = sum(b - a for a, b, _ in ran)
+    mid = len(ran) // 2
+    lines = ["CTAs that ran: %d of %d; kernel span (first start to last end): %.2f us" % (len(ran), len(spans), (t1 - t0) / 1e3),
+             "start after the first CTA's start, us: median %.2f, 90%% %.2f, max %.2f" % (
+                 starts[mid] / 1e3, starts[int(0.9 * (len(ran) - 1))] / 1e3, starts[-1] / 1e3),
+             "end before the last CTA's end, us: median %.2f, 90%% %.2f, max %.2f" % (
+                 ends[mid] / 1e3, ends[int(0.9 * (len(ran) - 1))] / 1e3, ends[-1] / 1e3),
+             "CTA life summed / kernel span: %.1f CTAs resident on average (the GPU has %d SMs)" % (busy / max(1, t1 - t0), sms),
+             "tiles per CTA: min %d, max %d, total %d" % (min(t for _, _, t in ran), max(t for _, _, t in ran), sum(t for _, _, t in ran))]
+    return "\n".join(lines)
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__.split("\n")[0])
     ap.add_argument("workload")
     ap.add_argument("--cta", type=int, default=0, help="blockIdx.x of the traced CTA")
     ap.add_argument("--tile", type=int, default=0, help="first of the CTA's two traced tiles")
+    ap.add_argument("--spans", action="store_true",
+                    help="instead of the role timeline: when every CTA of a (warm) launch started and ended")
     args = ap.parse_args(argv)
     import torch
     from . import binding, inputs
@@ -87,6 +111,22 @@ def main(argv=None):
     if st != binding.AVE_OK:
         raise RuntimeError("device status %d raw %#x" % (st, raw))
     L = binding.lib()
+    if args.spans:
+        n_ctas = 8192
+        L.ave_attn_trace_read_spans.argtypes = [ctypes.c_void_p, ctypes.c_int]
+        L.ave_attn_trace_read_spans.restype = ctypes.c_int
+        L.ave_attn_trace_clear_spans.restype = ctypes.c_int
+        for _ in range(3):   # the launch that is read is a warm one
+            if L.ave_attn_trace_clear_spans() != 0:
+                raise RuntimeError("ave_attn_trace_clear_spans failed")
+            binding.ave_attn_fwd(q, k, v, causal=w.causal, scale=w.scale)
+        sp = (ctypes.c_ulonglong * (3 * n_ctas))()
+        if L.ave_attn_trace_read_spans(sp, n_ctas) != 0:
+            raise RuntimeError("ave_attn_trace_read_spans failed")
+        vals = list(sp)
+        print(span_summary([tuple(vals[3 * i:3 * i + 3]) for i in range(n_ctas)],
+                           torch.cuda.get_device_properties(0).multi_processor_count))
+        return 0
     buf = (ctypes.c_longlong * (ROLES * ITERS * SLOTS))()
     L.ave_attn_trace_read.argtypes = [ctypes.c_void_p]
     L.ave_attn_trace_read.restype = ctypes.c_int
