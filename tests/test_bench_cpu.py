@@ -75,3 +75,15 @@ def test_timeline_decodes_the_stamp_array():
     assert ev[3] == (700, "LD ", "T0 Q0 issue")
     assert ev[4] == (1200, "SM1", "T1 epilogue done")
     assert t.events([0] * len(st)) == []
+
+
+def test_timeline_span_summary():
+    """Per-CTA (first ns, last ns, tiles) triples -> kernel span, how ragged the start and the end are, average
+    residency; CTAs whose index a running CTA took over have no start and are left out."""
+    from paper_2604_18616_b200 import timeline as t
+    txt = t.span_summary([(1000, 9000, 3), (1500, 8000, 2), (0, 0, 0), (2000, 9500, 4)], sms=4)
+    assert "CTAs that ran: 3 of 4" in txt and "8.50 us" in txt
+    assert "max 1.00" in txt and "max 1.50" in txt            # latest start, earliest end
+    assert "2.6 CTAs resident" in txt                         # (8000 + 6500 + 7500) / 8500
+    assert "min 2, max 4, total 9" in txt
+    assert t.span_summary([(0, 0, 0)] * 5) == "no CTA ran"
