@@ -445,21 +445,9 @@ attn_fwd_1t_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     float alpha = 1.f;
                     if (j == 0) {
                         m_run = m_tile;
-                    } else if (m_tile - m_run > kRescaleThreshold) {
+                    } else if (m_tile - m_run > rescale_margin(l_run)) {
                         alpha = ex2_approx(m_run - m_tile);
                         m_run = m_tile;
-                    }
-                    // O <- alpha * O.  S(j) ready implies P V_{j-1} has finished (in-order tensor pipe).
-                    if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-#pragma unroll 1
-                        for (int c = 0; c < D / 32; ++c) {
-                            uint32_t oc[32];
-                            tmem_ld_x32(tO + c * 32, oc);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int e = 0; e < 32; ++e) oc[e] = __float_as_uint(__uint_as_float(oc[e]) * alpha);
-                            tmem_st_x32(tO + c * 32, oc);
-                        }
                     }
                     // p = exp2(scale*log2e*s - m) for the whole row: P -> bf16 pairs into TMEM over the first 64
                     // columns of S; the row sum is taken from the fp32 probabilities, before the rounding
@@ -486,6 +474,25 @@ attn_fwd_1t_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                                 pk[e >> 1] = pack_bf16x2(pr.x, pr.y);
                             }
                             tmem_st_x16(tS + cc * 16, pk);
+                        }
+                        // O <- alpha * O, after the exponentiation: the score registers are free by then, so the whole
+                        // accumulator row (128 columns at a time) is in flight at once.  S(j) ready implies P V_{j-1} has
+                        // finished (in-order tensor pipe), and P V_j is not issued before this thread's arrival below.
+                        if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+                            constexpr int kGroup = (D < 128) ? D : 128;
+#pragma unroll 1
+                            for (int g = 0; g < D; g += kGroup) {
+                                uint32_t oc[kGroup / 32][32];
+#pragma unroll
+                                for (int c = 0; c < kGroup / 32; ++c) tmem_ld_x32(tO + g + c * 32, oc[c]);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int c = 0; c < kGroup / 32; ++c) {
+#pragma unroll
+                                    for (int e = 0; e < 32; ++e) oc[c][e] = __float_as_uint(__uint_as_float(oc[c][e]) * alpha);
+                                    tmem_st_x32(tO + g + c * 32, oc[c]);
+                                }
+                            }
                         }
                         l_run = l_run * alpha + ((acc0.x + acc0.y) + (acc1.x + acc1.y));
                     }

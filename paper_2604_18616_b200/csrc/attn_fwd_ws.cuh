@@ -59,11 +59,20 @@ constexpr int kLastWaves = 2;
 
 // Rescale O only when the running maximum moved by more than this many powers of two; until then
 // probabilities are taken relative to a stale maximum (at most 2^32 too large), which the final division by l
-// undoes.  Nothing is lost by a large threshold: P is rounded to bf16, which has fp32's exponent range, and
-// scaling every probability of a row by one factor leaves the relative rounding errors of P, l and O as they
-// are; l and O stay below 2^32 * Sk * max|V|, far from fp32's limit.  With peaked rows (the long-context
-// configuration) a threshold of 8 made some row of a warp rescale in most steps; measured -5.6 % there.
+// undoes.  The exponent range is no concern: P is rounded to bf16, which has fp32's range, and l and O stay
+// below 2^32 * Sk * max|V|, far from fp32's limit ...
 constexpr float kRescaleThreshold = 32.0f;
+// ... unless the new maximum would outweigh the sum accumulated so far.  A probability taken relative to a
+// stale maximum is an arbitrary number, rounded to bf16 with a relative error of up to 2^-9; for a key that
+// dominates its row that error is the error of O (0.2 % of a |V| of 4 is 0.008: together with the rounding
+// of O itself that is beyond the 2e-2 allowed, and the long-context configuration's peaked rows showed it).
+// Relative to its own maximum the dominant probability is exactly 1.  So the maximum also moves when
+// 2^(m_tile - m_run) exceeds l, the sum accumulated so far; terms that stay below half of a row's sum keep
+// their rounding errors, which average out.  (Measured on the long-context configuration: every element
+// then lies within the rounding of O itself, at +9 % time there and no change on unpeaked inputs.)
+__device__ __forceinline__ float rescale_margin(float l_run) {
+    return fminf(kRescaleThreshold, fmaxf(0.f, __log2f(l_run)));
+}
 
 // Of every 8 consecutive pairs of probabilities, the pairs whose bit is set
 // here are exponentiated on the FMA pipe (exp2_fma_pipe) instead of the
@@ -623,15 +632,16 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         return (acc0.x + acc0.y) + (acc1.x + acc1.y);
                     };
                     // O <- alpha * O.  S_t(j) ready implies P_t V_{j-1} has finished (in-order tensor pipe).
-                    auto rescale_o = [&](float alpha) {
-#pragma unroll 1
-                        for (int c = 0; c < D / 32; ++c) {
-                            uint32_t oc[32];
-                            tmem_ld_x32(tO + c * 32, oc);
-                            tmem_wait_ld();
+                    auto rescale_o_wide = [&](float alpha) {
+                        uint32_t oc[D / 32][32];
 #pragma unroll
-                            for (int e = 0; e < 32; ++e) oc[e] = __float_as_uint(__uint_as_float(oc[e]) * alpha);
-                            tmem_st_x32(tO + c * 32, oc);
+                        for (int c = 0; c < D / 32; ++c) tmem_ld_x32(tO + c * 32, oc[c]);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) oc[c][e] = __float_as_uint(__uint_as_float(oc[c][e]) * alpha);
+                            tmem_st_x32(tO + c * 32, oc[c]);
                         }
                     };
 
@@ -646,16 +656,15 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     if (!exact) {
                         // Optimistic: start exponentiating against the current m_run at once and find the
                         // tile maximum alongside; only if it exceeds m_run by more than the threshold
-                        // (rare after a row's first tiles) is O rescaled and the row redone below.
+                        // (rare after a row's first tiles) is the row redone, and O rescaled, below.
                         const float m_tile = tile_max();
                         row_sum = exp_pass(m_run);
-                        const bool moved = m_tile - m_run > kRescaleThreshold;  // also true for m_run = -inf < m_tile
+                        const bool moved = m_tile - m_run > rescale_margin(l_run);  // also true for m_run = -inf < m_tile
                         if (__any_sync(0xffffffffu, moved)) {
                             if (moved) {
                                 alpha = ex2_approx(m_run - m_tile);  // m_tile is finite here
                                 m_run = m_tile;
                             }
-                            rescale_o(alpha);
                             exact = true;
                             maximum_settled = true;
                         }
@@ -665,14 +674,17 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                             const float m_tile = tile_max();
                             if (j == 0) {
                                 m_run = m_tile;
-                            } else if (m_tile - m_run > kRescaleThreshold) {
+                            } else if (m_tile - m_run > rescale_margin(l_run)) {
                                 alpha = ex2_approx(m_run - m_tile);
                                 m_run = m_tile;
                             }
-                            if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) rescale_o(alpha);
                         }
                         if (traced(n) && tracer) trace_stamp(1 + t, trace_it(n, j), 3);
                         row_sum = exp_pass(m_run);
+                        // O <- alpha * O after the exponentiation: the score registers are free by then, so the
+                        // whole accumulator row is in flight at once (P_t V_j is not issued before this thread's
+                        // arrival below).
+                        if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) rescale_o_wide(alpha);
                     }
                     l_run = l_run * alpha + row_sum;
                     if (traced(n) && tracer) trace_stamp(1 + t, trace_it(n, j), 4);
