@@ -158,6 +158,27 @@ def test_peaked_and_drifting_scores_force_rescaling():
     parity.check_full(q.to(torch.bfloat16), k.flip(2).to(torch.bfloat16), v.to(torch.bfloat16), True, 0.05, "drift-rev")
 
 
+def test_dominant_keys_with_large_values_stay_within_the_rounding_of_o():
+    """Rows whose sum is dominated by one key (every 64th key scaled by 4, as in the long-context configuration)
+    and values large enough that |O| passes 4, where the rounding of O to bf16 alone is up to 0.0156: the
+    kernel has to add next to nothing there.  A dominant key's probability taken relative to a stale maximum
+    is rounded to bf16 with an error of up to 0.2 %, which is 0.01 of such an O (a kernel that keeps the stale
+    maximum there is 0.03 off on this input)."""
+    B, H, Hkv, S, D = 1, 4, 2, 2048, 128
+    g = torch.Generator().manual_seed(77)
+    q = torch.randn(B, H, S, D, generator=g)
+    k = torch.randn(B, Hkv, S, D, generator=g)
+    k[:, :, ::64, :] *= 4.0
+    v = torch.randn(B, Hkv, S, D, generator=g) * 1.4
+    q, k, v = q.to(torch.bfloat16), k.to(torch.bfloat16), v.to(torch.bfloat16)
+    scale = 1.0 / math.sqrt(D)
+    for causal in (True, False):
+        o_ref, lse_ref = oracle.attn_fwd(q, k, v, causal, scale)
+        assert np.abs(o_ref).max() > 4.0          # the case is what it claims to be
+        o, lse = parity.run_gpu(q, k, v, causal, scale)
+        parity.compare(o, lse, o_ref, lse_ref, "dominant keys, causal=%s" % causal)
+
+
 def test_gqa_equals_replicated_heads_bitwise():
     q, k, v = rand_qkv(13, 2, 8, 2, 300, 300, 128)
     o1, l1 = parity.run_gpu(q, k, v, True, 0.09)
