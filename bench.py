@@ -57,7 +57,15 @@ PER_WORKLOAD_DEFAULT = [
 ]
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel, from profiler captures of the
 # kernel as committed; a workload whose kernel has changed since its capture is absent (reported as null).
-NCU_DRAM_BYTES_PER_LAUNCH = {}
+NCU_DRAM_BYTES_PER_LAUNCH = {
+    "c2_mha_prefill": 325_227_136,        # profiles/attn_fwd_ws_c2_mha_prefill_ncu.md
+    "c3_gqa_prefill": 266_534_272,        # profiles/attn_fwd_ws_c3_gqa_prefill_ncu.md
+    "c4_long_context": 309_833_600,       # profiles/attn_fwd_ws_c4_long_context_ncu.md
+    "c5_wide_noncausal": 558_852_480,     # profiles/attn_fwd_ws_c5_wide_noncausal_ncu.md
+    "d256_gqa_prefill": 303_363_968,      # profiles/attn_fwd_1t_d256_gqa_prefill_ncu.md
+    "decode_mha_b8_k8192": 1_078_524_644, # profiles/attn_fwd_1t_decode_mha_b8_k8192_ncu.md
+    "gemm_n8192": 1_096_847_744,          # profiles/gemm_bf16_n8192_ncu.md
+}
 # Unit rates measured on this part (SM clocks per instruction): one M128xN128xK16 bf16 tcgen05.mma takes 64 clk,
 # an N = 64 one 47 clk; the exponential unit delivers 16 results per clock per SM.
 MMA_CLK_N128, MMA_CLK_N64, EX2_PER_CLK, N_SMS = 64.0, 47.0, 16.0, 148
